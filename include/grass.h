@@ -1,0 +1,154 @@
+/*
+ * grass.h -- C ABI of the B200 (sm_100a) gradient-compression library.
+ *
+ * The calls follow the problem statement of "GraSS: Scalable Data Attribution
+ * with Gradient Sparsification and Sparse Projection" (arXiv 2505.18976):
+ *
+ *   grass_compress               SJLT_k o Mask_k'      on dense per-sample gradients (Section 3.3.1)
+ *   factgrass_compress           SJLT_k o Mask_{k'_in (x) k'_out} for one linear layer (Section 3.3.2)
+ *   factgrass_compress_grouped   the same for many layers in one launch
+ *   grass_score                  all-pair inner products of compressed vectors (Section 2.1, attribute stage)
+ *
+ * Conventions (all calls):
+ *   - Pointers are DEVICE pointers unless the parameter is marked "host".  The caller owns every
+ *     buffer; the library allocates nothing and keeps no state between calls.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work is
+ *     enqueued on it and the call returns without synchronising, except where stated.
+ *   - Output buffers are OVERWRITTEN (the call zeroes them itself where its kernels accumulate).
+ *   - Arguments that can be checked on the host (null pointers, negative sizes, k == 0, s == 0,
+ *     k' > p, strides shorter than the row) are rejected with GRASS_ERR_INVALID_ARG before any
+ *     launch.  Launch failures return GRASS_ERR_CUDA.  Faults only visible on the device (a mask
+ *     index >= p, a bounded wait that expired) never trap or hang: the offending element is skipped
+ *     and a bit is OR-ed into *dev_status (nullable; the caller zeroes and reads it).
+ *   - Zero-size calls (n == 0, B == 0, T == 0 ...) are valid and leave a zeroed / untouched output.
+ *   - Mask index lists are uint32, strictly ascending, < p ("exactly one non-repetitive non-zero
+ *     entry per row" of the selection matrix, Section 3.2).  They are shared by all samples of a call.
+ *
+ * The sparse projection (Section 3.1) is defined by a seed, not by stored indices.  For input
+ * position j (position in the MASKED vector) and draw r < s:
+ *       H      = mix64(seed + 0x9E3779B97F4A7C15 * (j*s + r + 1))        (SplitMix64 stream)
+ *       bucket = ((H >> 32) * k) >> 32,   sign = (H & 1) ? -1 : +1
+ *       out[bucket] += sign * value / sqrt(s)
+ */
+#ifndef GRASS_H_
+#define GRASS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GRASS_OK = 0,
+    GRASS_ERR_INVALID_ARG = 1,
+    GRASS_ERR_BAD_MASK = 2,
+    GRASS_ERR_UNSUPPORTED = 3,
+    GRASS_ERR_CUDA = 4,
+    GRASS_ERR_TIMEOUT = 5
+} grass_status;
+
+typedef enum { GRASS_F32 = 0, GRASS_BF16 = 1 } grass_dtype;
+
+/* bits OR-ed into *dev_status by kernels */
+#define GRASS_DEV_BAD_INDEX 1u   /* a mask index was >= the row length; that element was skipped */
+#define GRASS_DEV_TIMEOUT   2u   /* a bounded on-device wait expired */
+
+/* SJLT_k with s non-zeros per column of the projection matrix (Section 3.1).  k >= 1, s >= 1. */
+typedef struct {
+    uint32_t k;
+    uint32_t s;
+    uint64_t seed;
+} grass_sjlt_spec;
+
+/*
+ * GraSS (Section 3.3.1): out[i, :] = SJLT_{k,s,seed}( g[i, idx[0..kprime)] ),  i in [0, n).
+ *   g        n x p, row-major, row stride `ld` elements (ld >= p), dtype `dt` (fp32 or bf16).
+ *   idx      kprime ascending coordinates (Random or Selective Mask, Section 3.2); NULL means the
+ *            identity mask and requires kprime == p (plain SJLT, the k' = p case of Section 3.3.1).
+ *   out      n x spec->k fp32, row stride ld_out >= k.  Overwritten.
+ *   The masked vector is never written to memory: gather and scatter-add are one kernel.
+ */
+grass_status grass_compress(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld,
+                            const uint32_t* idx, int64_t kprime, const grass_sjlt_spec* spec /*host*/,
+                            float* out, int64_t ld_out, uint32_t* dev_status, void* stream);
+
+/*
+ * FactGraSS for one linear layer (Section 3.3.2, stages 1-3; Eq. 2 with selection matrices):
+ *   out[b, :] = SJLT( vec( sum_t A[b,t,mask_in] (x) G[b,t,mask_out] ) ),  flat index a*kout + c.
+ *   A   B x T x d_in   layer inputs,            token-major contiguous, dtype dt (bf16; see below)
+ *   G   B x T x d_out  pre-activation gradients, token-major contiguous, same dtype
+ *   out B x spec->k fp32, row stride ld_out.  Overwritten.
+ * The kin x kout block is accumulated in fp32 on tensor cores and never reaches memory.
+ * dt == GRASS_F32 returns GRASS_ERR_UNSUPPORTED.
+ */
+grass_status factgrass_compress(const void* A, const void* G, grass_dtype dt, int32_t B, int32_t T,
+                                int32_t d_in, int32_t d_out, const uint32_t* mask_in, int32_t kin,
+                                const uint32_t* mask_out, int32_t kout,
+                                const grass_sjlt_spec* spec /*host*/, float* out, int64_t ld_out,
+                                uint32_t* dev_status, void* stream);
+
+/* One linear layer of a grouped call.  Layer l writes out[b, out_offset .. out_offset + spec.k). */
+typedef struct {
+    const void* A;
+    const void* G;
+    const uint32_t* mask_in;
+    const uint32_t* mask_out;
+    int32_t d_in, d_out;
+    int32_t kin, kout;
+    grass_sjlt_spec spec;
+    int64_t out_offset;
+} factgrass_layer;
+
+/*
+ * FactGraSS over L layers that share B, T, dtype and the output matrix (the layer-wise compression
+ * of Section 3.3.2: one compressed block per layer, concatenated per sample).
+ *   layers     host array of L descriptors (device pointers inside).  It is copied to `workspace`
+ *              on `stream`; the host array may be reused as soon as the call returns.
+ *   workspace  device scratch of at least factgrass_grouped_workspace_bytes(L) bytes, 256-byte
+ *              aligned, owned by the caller, in use until the work enqueued by this call has finished.
+ *   out        B x ld_out fp32; each layer's [out_offset, out_offset + k) range is overwritten,
+ *              ranges of different layers must not overlap.
+ */
+grass_status factgrass_compress_grouped(const factgrass_layer* layers /*host*/, int32_t L, grass_dtype dt,
+                                        int32_t B, int32_t T, float* out, int64_t ld_out,
+                                        void* workspace, size_t workspace_bytes,
+                                        uint32_t* dev_status, void* stream);
+size_t factgrass_grouped_workspace_bytes(int32_t L);
+
+/*
+ * Attribute-stage scores (Section 2.1): scores[i*ld_s + m] = <train[i, :], test[m, :]>.
+ *   train N x D, test M x D, fp32 row-major with strides ld_train, ld_test >= D.
+ *   scores N x M fp32 (train-major), row stride ld_s >= M.  Overwritten.  fp32 accumulation.
+ * These are raw inner products of compressed gradients; preconditioning is the caller's.
+ */
+grass_status grass_score(const float* train, int64_t N, int64_t ld_train, const float* test, int64_t M,
+                         int64_t ld_test, int64_t D, float* scores, int64_t ld_s, void* stream);
+
+/*
+ * The (bucket, sign) table of SJLT_{k,s,seed} for input positions [0, kprime), produced by the same
+ * device code the compress kernels use: bucket[j*s + r], sign[j*s + r] (+1 / -1).  Both are device
+ * buffers of kprime*s entries.  For tests and for callers that want to store the projection.
+ */
+grass_status grass_sjlt_table(const grass_sjlt_spec* spec /*host*/, int64_t kprime, uint32_t* bucket,
+                              int8_t* sign, void* stream);
+
+/*
+ * Checks a device index list: strictly ascending and every entry < p.  SYNCHRONISES `stream`.
+ * Returns GRASS_OK or GRASS_ERR_BAD_MASK.
+ */
+grass_status grass_validate_mask(const uint32_t* idx, int64_t kprime, int64_t p, void* stream);
+
+/*
+ * Random Mask (Section 3.2): kprime distinct coordinates of [0, p), uniform over subsets, ascending,
+ * written to the HOST array idx_host.  Deterministic in `seed`.  Runs on the CPU (set-up, not hot path).
+ */
+grass_status grass_random_mask_host(int64_t p, int64_t kprime, uint64_t seed, uint32_t* idx_host /*host*/);
+
+const char* grass_status_string(grass_status st);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRASS_H_ */

@@ -1,0 +1,237 @@
+"""Thin ctypes binding of ``libgrass_b200.so`` (declared in ``include/grass.h``).
+
+Argument marshalling only: every step of the compression path runs in the CUDA
+kernels behind the C ABI.  Functions take torch CUDA tensors (or raw integer
+device pointers) and enqueue on torch's current stream.  There is no CPU
+fallback: if the shared library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+SO_PATH = os.path.join(HERE, "libgrass_b200.so")
+
+GRASS_OK = 0
+STATUS = {0: "GRASS_OK", 1: "GRASS_ERR_INVALID_ARG", 2: "GRASS_ERR_BAD_MASK", 3: "GRASS_ERR_UNSUPPORTED",
+          4: "GRASS_ERR_CUDA", 5: "GRASS_ERR_TIMEOUT"}
+F32, BF16 = 0, 1
+DEV_BAD_INDEX, DEV_TIMEOUT = 1, 2
+
+EXPORTS = ("grass_compress", "factgrass_compress", "factgrass_compress_grouped",
+           "factgrass_grouped_workspace_bytes", "grass_score", "grass_sjlt_table", "grass_validate_mask",
+           "grass_random_mask_host", "grass_status_string")
+
+
+class GrassError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {STATUS.get(code, code)} ({lib().grass_status_string(code).decode()})")
+
+
+class SjltSpec(ctypes.Structure):
+    _fields_ = [("k", ctypes.c_uint32), ("s", ctypes.c_uint32), ("seed", ctypes.c_uint64)]
+
+
+class FactgrassLayer(ctypes.Structure):
+    _fields_ = [("A", ctypes.c_void_p), ("G", ctypes.c_void_p), ("mask_in", ctypes.c_void_p),
+                ("mask_out", ctypes.c_void_p), ("d_in", ctypes.c_int32), ("d_out", ctypes.c_int32),
+                ("kin", ctypes.c_int32), ("kout", ctypes.c_int32), ("spec", SjltSpec),
+                ("out_offset", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(SO_PATH):
+            raise ImportError(f"{SO_PATH} is missing: build it with `python -m paper_2505_18976_b200.build` "
+                              "(there is no CPU fallback)")
+        L = ctypes.CDLL(SO_PATH)
+        i64, i32, vp, st = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int
+        sp = ctypes.POINTER(SjltSpec)
+        L.grass_compress.restype = st
+        L.grass_compress.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, i64, sp, vp, i64, vp, vp]
+        L.factgrass_compress.restype = st
+        L.factgrass_compress.argtypes = [vp, vp, ctypes.c_int, i32, i32, i32, i32, vp, i32, vp, i32, sp, vp, i64, vp, vp]
+        L.factgrass_compress_grouped.restype = st
+        L.factgrass_compress_grouped.argtypes = [ctypes.POINTER(FactgrassLayer), i32, ctypes.c_int, i32, i32, vp, i64,
+                                                 vp, ctypes.c_size_t, vp, vp]
+        L.factgrass_grouped_workspace_bytes.restype = ctypes.c_size_t
+        L.factgrass_grouped_workspace_bytes.argtypes = [i32]
+        L.grass_score.restype = st
+        L.grass_score.argtypes = [vp, i64, i64, vp, i64, i64, i64, vp, i64, vp]
+        L.grass_sjlt_table.restype = st
+        L.grass_sjlt_table.argtypes = [sp, i64, vp, vp, vp]
+        L.grass_validate_mask.restype = st
+        L.grass_validate_mask.argtypes = [vp, i64, i64, vp]
+        L.grass_random_mask_host.restype = st
+        L.grass_random_mask_host.argtypes = [i64, i64, ctypes.c_uint64, vp]
+        L.grass_status_string.restype = ctypes.c_char_p
+        L.grass_status_string.argtypes = [st]
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != GRASS_OK:
+        raise GrassError(code, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _need_cuda(*ts) -> None:
+    for t in ts:
+        if t is not None and not isinstance(t, int) and not t.is_cuda:
+            raise ValueError("device tensors required (the library has no CPU path)")
+
+
+def grass_compress(g: torch.Tensor, idx: Optional[torch.Tensor], k: int, s: int, seed: int,
+                   out: Optional[torch.Tensor] = None, p: Optional[int] = None,
+                   dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """out[i] = SJLT_{k,s,seed}(g[i, idx]) for the rows of g (n x ld, fp32 or bf16).
+    idx: uint32/int32 CUDA tensor of ascending coordinates, or None for the identity mask."""
+    _need_cuda(g, idx, out, dev_status)
+    assert g.dim() == 2 and g.stride(1) == 1
+    n, ld = g.shape[0], g.stride(0) if g.shape[0] > 1 else g.shape[1]
+    p = g.shape[1] if p is None else p
+    kprime = p if idx is None else idx.numel()
+    if out is None:
+        out = torch.empty((n, k), dtype=torch.float32, device=g.device)
+    assert out.dtype == torch.float32 and out.stride(1) == 1
+    spec = SjltSpec(k, s, seed & 0xFFFFFFFFFFFFFFFF)
+    _check(lib().grass_compress(_ptr(g), _dt(g), n, p, ld, _ptr(idx), kprime, ctypes.byref(spec), _ptr(out),
+                                out.stride(0) if n > 1 else max(out.shape[1], k), _ptr(dev_status), _stream()),
+           "grass_compress")
+    return out
+
+
+def factgrass_compress(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, mask_out: torch.Tensor,
+                       k: int, s: int, seed: int, out: Optional[torch.Tensor] = None,
+                       dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """One linear layer: out[b] = SJLT(vec(sum_t A[b,t,mask_in] (x) G[b,t,mask_out]))."""
+    _need_cuda(A, G, mask_in, mask_out, out, dev_status)
+    assert A.is_contiguous() and G.is_contiguous() and A.dim() == 3 and G.dim() == 3
+    B, T, d_in = A.shape
+    d_out = G.shape[2]
+    assert G.shape[:2] == (B, T)
+    if out is None:
+        out = torch.empty((B, k), dtype=torch.float32, device=A.device)
+    spec = SjltSpec(k, s, seed & 0xFFFFFFFFFFFFFFFF)
+    _check(lib().factgrass_compress(_ptr(A), _ptr(G), _dt(A), B, T, d_in, d_out, _ptr(mask_in), mask_in.numel(),
+                                    _ptr(mask_out), mask_out.numel(), ctypes.byref(spec), _ptr(out),
+                                    out.stride(0) if B > 1 else max(out.shape[1], k), _ptr(dev_status), _stream()),
+           "factgrass_compress")
+    return out
+
+
+class GroupedLayers:
+    """Host-side descriptor table for factgrass_compress_grouped; keeps the tensors alive."""
+
+    def __init__(self, layers: Sequence[dict]):
+        """layers: dicts with A, G, mask_in, mask_out (CUDA tensors), k, s, seed, out_offset."""
+        self.keep = list(layers)
+        self.L = len(layers)
+        self.array = (FactgrassLayer * max(self.L, 1))()
+        for i, l in enumerate(layers):
+            _need_cuda(l["A"], l["G"], l["mask_in"], l["mask_out"])
+            e = self.array[i]
+            e.A, e.G = l["A"].data_ptr(), l["G"].data_ptr()
+            e.mask_in, e.mask_out = l["mask_in"].data_ptr(), l["mask_out"].data_ptr()
+            e.d_in, e.d_out = l["A"].shape[-1], l["G"].shape[-1]
+            e.kin, e.kout = l["mask_in"].numel(), l["mask_out"].numel()
+            e.spec = SjltSpec(l["k"], l["s"], l["seed"] & 0xFFFFFFFFFFFFFFFF)
+            e.out_offset = l["out_offset"]
+        self.dtype = _dt(layers[0]["A"]) if layers else BF16
+        self.B, self.T = (layers[0]["A"].shape[0], layers[0]["A"].shape[1]) if layers else (0, 0)
+
+
+def factgrass_grouped_workspace_bytes(L: int) -> int:
+    return int(lib().factgrass_grouped_workspace_bytes(L))
+
+
+def factgrass_compress_grouped(group: GroupedLayers, out: torch.Tensor, workspace: torch.Tensor,
+                               dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """All layers of ``group`` in one launch; layer l fills out[:, off_l : off_l + k_l]."""
+    _need_cuda(out, workspace, dev_status)
+    assert out.dtype == torch.float32 and out.stride(1) == 1
+    _check(lib().factgrass_compress_grouped(group.array, group.L, group.dtype, group.B, group.T, _ptr(out),
+                                            out.stride(0) if out.shape[0] > 1 else out.shape[1], _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _ptr(dev_status),
+                                            _stream()), "factgrass_compress_grouped")
+    return out
+
+
+def grass_score(train: torch.Tensor, test: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """scores[i, m] = <train[i], test[m]> (fp32)."""
+    _need_cuda(train, test, out)
+    assert train.dtype == torch.float32 and test.dtype == torch.float32
+    assert train.stride(1) == 1 and test.stride(1) == 1
+    N, D = train.shape
+    M = test.shape[0]
+    assert test.shape[1] == D
+    if out is None:
+        out = torch.empty((N, M), dtype=torch.float32, device=train.device)
+    _check(lib().grass_score(_ptr(train), N, train.stride(0) if N > 1 else D, _ptr(test), M,
+                             test.stride(0) if M > 1 else D, D, _ptr(out), out.stride(0) if N > 1 else M,
+                             _stream()), "grass_score")
+    return out
+
+
+def grass_sjlt_table(k: int, s: int, seed: int, kprime: int, device="cuda"):
+    """(bucket uint32, sign int8) of length kprime*s, computed by the device hash code."""
+    bucket = torch.empty(kprime * s, dtype=torch.int32, device=device)
+    sign = torch.empty(kprime * s, dtype=torch.int8, device=device)
+    spec = SjltSpec(k, s, seed & 0xFFFFFFFFFFFFFFFF)
+    _check(lib().grass_sjlt_table(ctypes.byref(spec), kprime, _ptr(bucket), _ptr(sign), _stream()),
+           "grass_sjlt_table")
+    return bucket, sign
+
+
+def grass_validate_mask(idx: torch.Tensor, p: int) -> bool:
+    """True if idx (CUDA uint32/int32) is strictly ascending and < p.  Synchronises."""
+    _need_cuda(idx)
+    code = lib().grass_validate_mask(_ptr(idx), idx.numel(), p, _stream())
+    if code == 2:
+        return False
+    _check(code, "grass_validate_mask")
+    return True
+
+
+def grass_random_mask_host(p: int, kprime: int, seed: int) -> np.ndarray:
+    """Random Mask indices (ascending uint32 numpy array), sampled on the host by the library."""
+    idx = np.empty(kprime, dtype=np.uint32)
+    _check(lib().grass_random_mask_host(p, kprime, seed & 0xFFFFFFFFFFFFFFFF,
+                                        idx.ctypes.data_as(ctypes.c_void_p)), "grass_random_mask_host")
+    return idx
+
+
+def mask_to_device(idx: np.ndarray, device="cuda") -> torch.Tensor:
+    """uint32 index list -> CUDA tensor holding the same 32-bit patterns."""
+    return torch.from_numpy(np.ascontiguousarray(idx, dtype=np.uint32).view(np.int32)).to(device)

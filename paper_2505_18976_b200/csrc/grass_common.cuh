@@ -1,0 +1,70 @@
+// Shared device-side pieces of the sm_100a compression kernels: the seed-defined
+// SJLT hash (bucket, sign) recomputed in registers, bf16 helpers, launch checks.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/grass.h"
+
+namespace grass {
+
+constexpr uint64_t kGolden = 0x9E3779B97F4A7C15ULL;
+
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t x)
+{
+    x ^= x >> 30;
+    x *= 0xBF58476D1CE4E5B9ULL;
+    x ^= x >> 27;
+    x *= 0x94D049BB133111EBULL;
+    x ^= x >> 31;
+    return x;
+}
+
+// Hash of counter c = j*s + r + 1 under `seed` (Section 3.1: the random output
+// coordinate and sign that input position j draws).
+__host__ __device__ __forceinline__ uint64_t sjlt_hash_counter(uint64_t seed, uint64_t counter)
+{
+    return mix64(seed + kGolden * counter);
+}
+
+__host__ __device__ __forceinline__ uint32_t sjlt_bucket(uint64_t h, uint32_t k)
+{
+#ifdef __CUDA_ARCH__
+    return __umulhi((uint32_t)(h >> 32), k);
+#else
+    return (uint32_t)(((h >> 32) * (uint64_t)k) >> 32);
+#endif
+}
+
+// value with the hash's sign applied: flips the fp32 sign bit when H is odd.
+__device__ __forceinline__ float sjlt_signed(uint64_t h, float v)
+{
+    return __uint_as_float(__float_as_uint(v) ^ ((uint32_t)h << 31));
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b)
+{
+    return __uint_as_float((uint32_t)b << 16);
+}
+
+template <typename T> struct elem;
+template <> struct elem<float> {
+    static __device__ __forceinline__ float load(const float* p) { return __ldg(p); }
+};
+template <> struct elem<__nv_bfloat16> {
+    static __device__ __forceinline__ float load(const __nv_bfloat16* p)
+    {
+        return bf16_bits_to_float(__ldg(reinterpret_cast<const unsigned short*>(p)));
+    }
+};
+
+inline grass_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? GRASS_OK : GRASS_ERR_CUDA; }
+
+inline grass_status launch_status()
+{
+    return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace grass

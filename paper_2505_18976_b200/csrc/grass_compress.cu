@@ -1,0 +1,209 @@
+// grass_compress: Mask_k' gather fused with the SJLT_k scatter-add (GraSS, Section 3.3.1).
+//
+// One CTA owns S samples and a contiguous range of masked positions j.  Each thread reads the
+// mask index of its j once, derives (bucket, sign) once from the seed, and applies them to the S
+// samples: S independent gathered loads per j are in flight together, consecutive lanes hold
+// consecutive (ascending) indices so the loads of a warp fall into the fewest 32-byte sectors.
+// Non-zero values are added into a per-sample k-bin accumulator in shared memory; exact zeros are
+// skipped (the input sparsity the paper's Section 3.1 builds on).  Bins are flushed with coalesced
+// stores, or with global reductions when the j range of a sample is split over several CTAs.
+#include "grass_common.cuh"
+
+#include <cstdlib>
+
+namespace grass {
+
+constexpr int kThreads = 256;
+
+template <typename T, int S, int U, bool S1>
+__global__ void __launch_bounds__(kThreads)
+grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
+                      const uint32_t* __restrict__ idx, int64_t kprime, uint32_t k, uint32_t s,
+                      uint64_t seed, float scale, float* __restrict__ out, int64_t ld_out,
+                      int64_t j_per_cta, int accumulate, int use_smem, uint32_t* dev_status)
+{
+    extern __shared__ float bins[];  // S * k when use_smem
+    const int tid = threadIdx.x;
+    const int64_t i0 = (int64_t)blockIdx.x * S;
+    const int ns = (int)((n - i0) < (int64_t)S ? (n - i0) : (int64_t)S);
+    const int64_t j0 = (int64_t)blockIdx.y * j_per_cta;
+    const int64_t j1 = (j0 + j_per_cta) < kprime ? (j0 + j_per_cta) : kprime;
+
+    if (use_smem) {
+        for (uint32_t i = tid; i < (uint32_t)S * k; i += kThreads) bins[i] = 0.0f;
+        __syncthreads();
+    }
+
+    const T* rows[S];
+#pragma unroll
+    for (int si = 0; si < S; ++si) rows[si] = g + (i0 + (si < ns ? si : 0)) * ld;
+
+    bool bad = false;
+    for (int64_t jb = j0 + tid; jb < j1; jb += (int64_t)kThreads * U) {
+        uint32_t col[U];
+        bool ok[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t j = jb + (int64_t)u * kThreads;
+            ok[u] = j < j1;
+            uint32_t c = 0;
+            if (ok[u]) c = idx ? __ldg(idx + j) : (uint32_t)j;
+            if ((int64_t)c >= p) { bad = bad || ok[u]; ok[u] = false; c = 0; }
+            col[u] = c;
+        }
+        float v[U][S];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+#pragma unroll
+            for (int si = 0; si < S; ++si)
+                v[u][si] = (ok[u] && si < ns) ? elem<T>::load(rows[si] + col[u]) : 0.0f;
+
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (!ok[u]) continue;
+            const uint64_t j = (uint64_t)(jb + (int64_t)u * kThreads);
+            const uint32_t draws = S1 ? 1u : s;
+            for (uint32_t r = 0; r < draws; ++r) {
+                const uint64_t h = sjlt_hash_counter(seed, S1 ? (j + 1) : (j * s + r + 1));
+                const uint32_t b = sjlt_bucket(h, k);
+#pragma unroll
+                for (int si = 0; si < S; ++si) {
+                    const float x = v[u][si];
+                    if (x != 0.0f) {
+                        const float sx = S1 ? sjlt_signed(h, x) : sjlt_signed(h, x) * scale;
+                        if (use_smem) atomicAdd(&bins[(uint32_t)si * k + b], sx);
+                        else atomicAdd(out + (i0 + si) * ld_out + b, sx);
+                    }
+                }
+            }
+        }
+    }
+    if (bad && dev_status) atomicOr(dev_status, GRASS_DEV_BAD_INDEX);
+
+    if (use_smem) {
+        __syncthreads();
+        for (int si = 0; si < ns; ++si) {
+            float* dst = out + (i0 + si) * ld_out;
+            const float* src = bins + (uint32_t)si * k;
+            if (accumulate) {
+                for (uint32_t i = tid; i < k; i += kThreads) {
+                    const float x = src[i];
+                    if (x != 0.0f) atomicAdd(dst + i, x);
+                }
+            } else {
+                for (uint32_t i = tid; i < k; i += kThreads) dst[i] = src[i];
+            }
+        }
+    }
+}
+
+struct CompressPlan {
+    int S;
+    int jsplit;
+    int use_smem;
+};
+
+static int env_int(const char* name, int dflt)
+{
+    const char* v = std::getenv(name);
+    return v ? std::atoi(v) : dflt;
+}
+
+static CompressPlan plan_compress(int64_t n, int64_t kprime, uint32_t k, int sm_count)
+{
+    CompressPlan pl;
+    const size_t bin_bytes = (size_t)k * sizeof(float);
+    const size_t smem_cap = 200 * 1024;
+    pl.use_smem = bin_bytes <= smem_cap;
+    // samples per CTA: amortise the hash over S gathered loads, keep >= 3 CTAs per SM resident
+    int S = 4;
+    while (S > 1 && (bin_bytes * S > 64 * 1024 || (n + S - 1) / S < sm_count)) S >>= 1;
+    if (!pl.use_smem) S = 1;
+    S = env_int("GRASS_COMPRESS_S", S);
+    if (S != 1 && S != 2 && S != 4 && S != 8) S = 1;
+    while (S > 1 && pl.use_smem && bin_bytes * S > smem_cap) S >>= 1;
+    pl.S = S;
+    const int64_t groups = (n + S - 1) / S;
+    const int64_t target = (int64_t)sm_count * 4;
+    int64_t js = (target + groups - 1) / (groups > 0 ? groups : 1);
+    // keep at least 8 positions per thread per CTA so the bin zero/flush is amortised
+    const int64_t max_js = kprime / (kThreads * 8) > 0 ? kprime / (kThreads * 8) : 1;
+    if (js > max_js) js = max_js;
+    if (js < 1) js = 1;
+    js = env_int("GRASS_COMPRESS_JSPLIT", (int)js);
+    if (js < 1) js = 1;
+    if (js > 65535) js = 65535;
+    pl.jsplit = (int)js;
+    return pl;
+}
+
+template <typename T, int S, int U>
+static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld, const uint32_t* idx,
+                                    int64_t kprime, const grass_sjlt_spec& sp, float* out, int64_t ld_out,
+                                    const CompressPlan& pl, uint32_t* dev_status, cudaStream_t st)
+{
+    const int64_t groups = (n + S - 1) / S;
+    const int64_t j_per_cta = (kprime + pl.jsplit - 1) / pl.jsplit;
+    const int accumulate = (pl.jsplit > 1 || !pl.use_smem) ? 1 : 0;
+    const size_t smem = pl.use_smem ? (size_t)S * sp.k * sizeof(float) : 0;
+    const float scale = 1.0f / sqrtf((float)sp.s);
+    dim3 grid((unsigned)groups, (unsigned)pl.jsplit);
+    auto launch = [&](auto kern) -> grass_status {
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return GRASS_ERR_CUDA;
+        }
+        kern<<<grid, kThreads, smem, st>>>(g, n, p, ld, idx, kprime, sp.k, sp.s, sp.seed, scale, out, ld_out,
+                                           j_per_cta, accumulate, pl.use_smem, dev_status);
+        return launch_status();
+    };
+    if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true>);
+    return launch(grass_compress_kernel<T, S, U, false>);
+}
+
+template <typename T>
+static grass_status dispatch_compress(const T* g, int64_t n, int64_t p, int64_t ld, const uint32_t* idx,
+                                      int64_t kprime, const grass_sjlt_spec& sp, float* out, int64_t ld_out,
+                                      uint32_t* dev_status, cudaStream_t st)
+{
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    const CompressPlan pl = plan_compress(n, kprime, sp.k, sms);
+    if (pl.jsplit > 1 || !pl.use_smem) {
+        cudaError_t e = cudaMemset2DAsync(out, (size_t)ld_out * sizeof(float), 0, (size_t)sp.k * sizeof(float),
+                                          (size_t)n, st);
+        if (e != cudaSuccess) return GRASS_ERR_CUDA;
+    }
+    switch (pl.S) {
+        case 8: return launch_compress<T, 8, 2>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
+        case 4: return launch_compress<T, 4, 4>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
+        case 2: return launch_compress<T, 2, 4>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
+        default: return launch_compress<T, 1, 4>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
+    }
+}
+
+}  // namespace grass
+
+extern "C" grass_status grass_compress(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld,
+                                       const uint32_t* idx, int64_t kprime, const grass_sjlt_spec* spec,
+                                       float* out, int64_t ld_out, uint32_t* dev_status, void* stream)
+{
+    if (!spec || spec->k == 0 || spec->s == 0) return GRASS_ERR_INVALID_ARG;
+    if (n < 0 || p < 0 || kprime < 0 || kprime > p || ld < p || ld_out < (int64_t)spec->k) return GRASS_ERR_INVALID_ARG;
+    if (p >= 0xFFFFFFFFLL) return GRASS_ERR_INVALID_ARG;
+    if (!idx && kprime != p) return GRASS_ERR_INVALID_ARG;
+    if (dt != GRASS_F32 && dt != GRASS_BF16) return GRASS_ERR_UNSUPPORTED;
+    if (n == 0) return GRASS_OK;
+    if (!out || (!g && kprime > 0)) return GRASS_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (kprime == 0) {
+        return grass::cuda_ok(cudaMemset2DAsync(out, (size_t)ld_out * sizeof(float), 0,
+                                                (size_t)spec->k * sizeof(float), (size_t)n, st));
+    }
+    if (dt == GRASS_F32)
+        return grass::dispatch_compress<float>((const float*)g, n, p, ld, idx, kprime, *spec, out, ld_out,
+                                               dev_status, st);
+    return grass::dispatch_compress<__nv_bfloat16>((const __nv_bfloat16*)g, n, p, ld, idx, kprime, *spec, out,
+                                                   ld_out, dev_status, st);
+}

@@ -1,0 +1,375 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by
+element, on the same seeded inputs.  Indices, buckets and signs bit-exact; values within
+the tolerance rule of tests/parity.py."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from parity import check_close, max_bin_load
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32, TOL_BF16 = 1e-4, 2e-2
+EPS_TC = 2.0 ** -23
+
+
+@pytest.fixture(scope="module")
+def G():
+    import paper_2505_18976_b200 as g
+    g.lib()
+    return g
+
+
+@pytest.fixture(scope="module")
+def W():
+    from paper_2505_18976_b200 import workloads
+    return workloads
+
+
+def _dev_mask(G, idx):
+    return G.mask_to_device(idx)
+
+
+# ------------------------------------------------------------------ hash, bit-exact
+
+@pytest.mark.parametrize("k,s,seed,kp", [(2048, 1, 0x5EED + 1, 8192), (4096, 1, 0x5EED + 2, 65536),
+                                         (1000003, 3, 7, 5000), (1, 2, 9, 100), (4294967295, 1, 2 ** 64 - 1, 4096)])
+def test_device_hash_table_bit_exact(G, oracle_mod, k, s, seed, kp):
+    b, sg = G.grass_sjlt_table(k, s, seed, kp)
+    ob, osg = oracle_mod.sjlt_table(k, s, seed, kp)
+    assert np.array_equal(b.cpu().numpy().view(np.uint32), ob)
+    assert np.array_equal(sg.cpu().numpy(), osg)
+
+
+def test_one_hot_through_grass_compress_reads_the_table(G, oracle_mod):
+    """e_j in -> sign(j) e_{bucket(j)} out, through the compress kernel itself."""
+    p, k, seed = 1536, 257, 0xBEEF
+    out = G.grass_compress(torch.eye(p, device="cuda"), None, k, 1, seed).cpu().numpy()
+    ob, osg = oracle_mod.sjlt_table(k, 1, seed, p)
+    expect = np.zeros((p, k), dtype=np.float32)
+    expect[np.arange(p), ob] = osg
+    assert np.array_equal(out, expect)
+
+
+def test_one_hot_through_factgrass_reads_the_table(G, oracle_mod):
+    """T = 1, A = e_a, G = e_c: the only non-zero block entry sits at q = a*kout + c."""
+    kin, kout, k, seed = 24, 40, 97, 11
+    d_in, d_out = 64, 96
+    mi = oracle_mod.random_mask(d_in, kin, 1)
+    mo = oracle_mod.random_mask(d_out, kout, 2)
+    pairs = [(0, 0), (3, 7), (23, 39), (10, 0), (0, 39)]
+    A = torch.zeros(len(pairs), 1, d_in, dtype=torch.bfloat16, device="cuda")
+    Gt = torch.zeros(len(pairs), 1, d_out, dtype=torch.bfloat16, device="cuda")
+    for n, (a, c) in enumerate(pairs):
+        A[n, 0, int(mi[a])] = 1.0
+        Gt[n, 0, int(mo[c])] = 1.0
+    out = G.factgrass_compress(A, Gt, _dev_mask(G, mi), _dev_mask(G, mo), k, 1, seed).cpu().numpy()
+    ob, osg = oracle_mod.sjlt_table(k, 1, seed, kin * kout)
+    for n, (a, c) in enumerate(pairs):
+        e = np.zeros(k, dtype=np.float32)
+        e[ob[a * kout + c]] = osg[a * kout + c]
+        assert np.array_equal(out[n], e), (a, c)
+
+
+# ------------------------------------------------------------------ grass_compress
+
+def _grass_case(G, W, oracle_mod, n, p, kprime, k, s=1, dtype=torch.float32, ld=None, identity=False,
+                zero_prob=0.8, dist="normal", scale=1.0, seed=0, data_seed=5):
+    g = W.dense_gradients(n, p, zero_prob, dist, scale, data_seed, device="cuda", dtype=dtype, ld=ld)
+    idx = None if identity else oracle_mod.random_mask(p, kprime, seed)
+    didx = None if identity else _dev_mask(G, idx)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = G.grass_compress(g, didx, k, s, seed + 99, p=p, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    host = W.bits_of(g)
+    ref, absum = oracle_mod.grass(host, idx, k, s, seed + 99, dtype="f32" if dtype == torch.float32 else "bf16", p=p)
+    kp = p if identity else kprime
+    ob, _ = oracle_mod.sjlt_table(k, s, seed + 99, kp)
+    chain = max_bin_load(ob, k) + 16
+    return check_close(out.cpu().numpy(), ref, absum, TOL_F32, chain,
+                       what=f"grass n={n} p={p} k'={kp} k={k} s={s}")
+
+
+@pytest.mark.parametrize("n,p,kprime,k", [
+    (64, 65_536, 8_192, 2_048),        # config 1 scaled in n
+    (16, 1 << 20, 16_384, 4_096),      # config 2 scaled in p and k'
+    (7, 10_007, 1_237, 333),           # nothing a multiple of anything
+    (3, 4_096, 4_096, 64),             # mask covers every coordinate
+    (5, 70_000, 33, 4_096),            # fewer masked coordinates than a warp
+    (9, 300_000, 50_000, 60_000),      # k too large for shared-memory bins: global path
+    (1, 50_000, 9_999, 1),             # single output bin
+])
+def test_grass_compress_parity(G, W, oracle_mod, n, p, kprime, k):
+    _grass_case(G, W, oracle_mod, n, p, kprime, k)
+
+
+@pytest.mark.parametrize("s", [2, 4])
+def test_grass_compress_s_gt_1(G, W, oracle_mod, s):
+    _grass_case(G, W, oracle_mod, 6, 20_000, 5_000, 512, s=s)
+
+
+def test_grass_compress_identity_mask_and_stride(G, W, oracle_mod):
+    _grass_case(G, W, oracle_mod, 10, 65_536, 65_536, 2_048, identity=True)
+    _grass_case(G, W, oracle_mod, 5, 9_001, 700, 100, ld=9_016)                  # ld > p, tail is NaN
+    _grass_case(G, W, oracle_mod, 5, 9_001, 9_001, 100, ld=9_016, identity=True)
+
+
+def test_grass_compress_bf16_input(G, W, oracle_mod):
+    _grass_case(G, W, oracle_mod, 12, 100_000, 10_000, 1_024, dtype=torch.bfloat16)
+
+
+def test_grass_compress_student_t(G, W, oracle_mod):
+    _grass_case(G, W, oracle_mod, 8, 1 << 18, 1 << 14, 4_096, zero_prob=0.7, dist="student_t3", scale=1e-2)
+
+
+@pytest.mark.parametrize("S,js", [(1, 1), (2, 3), (4, 7), (8, 2)])
+def test_grass_compress_launch_shapes(G, W, oracle_mod, monkeypatch, S, js):
+    """Every (samples per CTA, position split) plan gives the same answer."""
+    monkeypatch.setenv("GRASS_COMPRESS_S", str(S))
+    monkeypatch.setenv("GRASS_COMPRESS_JSPLIT", str(js))
+    _grass_case(G, W, oracle_mod, 11, 40_000, 9_000, 1_000)
+
+
+def test_grass_compress_special_values(G, oracle_mod):
+    """All-zero rows give exact zeros; NaN / Inf reach exactly the bins they hash to."""
+    n, p, k, seed = 4, 5_000, 64, 3
+    g = torch.zeros(n, p, device="cuda")
+    g[1, 17] = float("nan")
+    g[2, 4_000] = float("inf")
+    g[3, :] = 1.0
+    out = G.grass_compress(g, None, k, 1, seed).cpu().numpy()
+    ob, osg = oracle_mod.sjlt_table(k, 1, seed, p)
+    assert np.all(out[0] == 0)
+    assert np.isnan(out[1, ob[17]]) and np.all(np.delete(out[1], ob[17]) == 0)
+    assert np.isinf(out[2, ob[4_000]]) and out[2, ob[4_000]] == osg[4_000] * np.inf
+    assert np.array_equal(out[3], np.bincount(ob, weights=osg.astype(np.float64), minlength=k).astype(np.float32))
+
+
+def test_grass_compress_empty_and_errors(G, oracle_mod):
+    out = G.grass_compress(torch.empty(0, 100, device="cuda"), None, 8, 1, 0)
+    assert out.shape == (0, 8)
+    # k' = 0: output zeroed
+    idx = torch.empty(0, dtype=torch.int32, device="cuda")
+    o = torch.full((3, 8), 7.0, device="cuda")
+    G.grass_compress(torch.ones(3, 100, device="cuda"), idx, 8, 1, 0, out=o)
+    assert torch.all(o == 0)
+    # an index >= p (planted on the host) is skipped and flagged, never dereferenced
+    p, k = 1_000, 16
+    idxh = oracle_mod.random_mask(p, 50, 1)
+    bad = idxh.copy()
+    bad[-1] = 2_000_000_000
+    g = torch.randn(2, p, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = G.grass_compress(g, G.mask_to_device(bad), k, 1, 5, dev_status=st).cpu().numpy()
+    assert int(st.item()) & 1
+    ref_in = g.cpu().numpy().copy()
+    ref_in[:, idxh[-1]] = 0        # same as dropping the last masked position
+    ref, absum = oracle_mod.grass(ref_in, idxh, k, 1, 5)
+    check_close(got, ref, absum, TOL_F32, 32, what="bad index skipped")
+    assert not G.grass_validate_mask(G.mask_to_device(bad), p)
+    assert G.grass_validate_mask(G.mask_to_device(idxh), p)
+    dup = idxh.copy()
+    dup[10] = dup[9]
+    assert not G.grass_validate_mask(G.mask_to_device(dup), p)
+    with pytest.raises(G.GrassError):
+        G.grass_compress(g, G.mask_to_device(idxh), 0, 1, 5)
+
+
+def test_grass_compress_run_to_run(G, W, oracle_mod):
+    """Float atomics reorder sums: repeated runs agree to a few ulps of the bin's mass."""
+    g = W.dense_gradients(32, 100_000, 0.5, "normal", 1.0, 3, device="cuda")
+    idx = _dev_mask(G, oracle_mod.random_mask(100_000, 20_000, 0))
+    a = G.grass_compress(g, idx, 512, 1, 1).cpu().numpy().astype(np.float64)
+    for _ in range(3):
+        b = G.grass_compress(g, idx, 512, 1, 1).cpu().numpy().astype(np.float64)
+        assert np.max(np.abs(a - b)) <= 64 * 2.0 ** -24 * np.abs(a).max() * 8
+
+
+# ------------------------------------------------------------------ factgrass_compress
+
+def _fact_cfg(W, **kw):
+    base = dict(name="t", layers=(W.LinearLayer("l", 96, 160),), B=3, T=70, kin=24, kout=40, k=97, s=1,
+                g_dist="normal", g_scale=1e-3, pad_frac=0.0, data_seed=21, mask_seed=4, hash_seed=77)
+    base.update(kw)
+    return W.FactGrassWorkload(**base)
+
+
+def _fact_case(G, W, oracle_mod, cfg, l=0, grouped=False):
+    lay = cfg.layers[l]
+    A, Gt = W.layer_io(cfg, l, device="cuda")
+    s_in, s_out = W.layer_mask_seeds(cfg, l)
+    mi = oracle_mod.random_mask(lay.d_in, cfg.kin, s_in)
+    mo = oracle_mod.random_mask(lay.d_out, cfg.kout, s_out)
+    seed = W.layer_hash_seed(cfg, l)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = G.factgrass_compress(A, Gt, _dev_mask(G, mi), _dev_mask(G, mo), cfg.k, cfg.s, seed, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    ref, absum = oracle_mod.factgrass(W.bits_of(A), W.bits_of(Gt), mi, mo, cfg.k, cfg.s, seed)
+    ob, _ = oracle_mod.sjlt_table(cfg.k, cfg.s, seed, cfg.kin * cfg.kout)
+    chain = cfg.T + max_bin_load(ob, cfg.k) + 64
+    return check_close(out.cpu().numpy(), ref, absum, TOL_BF16, chain, eps=EPS_TC,
+                       what=f"factgrass {lay} B={cfg.B} T={cfg.T} k'={cfg.kin}x{cfg.kout} k={cfg.k}")
+
+
+@pytest.mark.parametrize("kw", [
+    dict(),                                                          # odd sizes, one 64x64 tile
+    dict(kin=5, kout=4, k=7, T=1),                                   # one token, tiny block
+    dict(kin=64, kout=64, k=1024, T=200, B=4),                       # configs 4/5 tile, ragged token tail
+    dict(kin=96, kout=160, k=4096, T=33),                            # mask = every coordinate; 128 tile; 2 column tiles
+    dict(layers=None, kin=128, kout=128, k=4096, T=130, B=3),        # config 3 tile
+    dict(layers=None, kin=130, kout=260, k=5000, T=64, B=2),         # several block tiles in both directions
+    dict(kin=24, kout=40, k=50_000, T=40),                           # k too large for shared-memory bins
+    dict(kin=24, kout=40, k=97, s=2),                                # two draws per position
+    dict(kin=64, kout=64, k=256, T=300, pad_frac=0.2, g_dist="laplace"),
+])
+def test_factgrass_parity(G, W, oracle_mod, kw):
+    kw = dict(kw)
+    if "layers" in kw and kw["layers"] is None:
+        kw["layers"] = (W.LinearLayer("l", 768, 3072),)
+    _fact_case(G, W, oracle_mod, _fact_cfg(W, **kw))
+
+
+@pytest.mark.parametrize("chunk", [32, 64, 1 << 20])
+def test_factgrass_token_chunking(G, W, oracle_mod, monkeypatch, chunk):
+    """Splitting the token sum over CTAs (linearity of SJLT) does not change the result."""
+    monkeypatch.setenv("FACTGRASS_CHUNK", str(chunk))
+    _fact_case(G, W, oracle_mod, _fact_cfg(W, T=250, kin=64, kout=64, k=512))
+
+
+def test_factgrass_scaled_configs(G, W, oracle_mod):
+    c3 = dataclasses.replace(W.CONFIG3, B=4, T=256)
+    _fact_case(G, W, oracle_mod, c3)
+    c4 = dataclasses.replace(W.CONFIG4, B=2, T=256)
+    for l in (0, 1, 3):
+        _fact_case(G, W, oracle_mod, c4, l=l)
+    c5 = dataclasses.replace(W.CONFIG5, B=1, T=256)
+    for l in (1, 4, 6):
+        _fact_case(G, W, oracle_mod, c5, l=l)
+
+
+def test_factgrass_padding_tokens_change_nothing(G, W, oracle_mod):
+    cfg = _fact_cfg(W, T=64, kin=64, kout=64, k=512)
+    A, Gt = W.layer_io(cfg, 0, device="cuda")
+    mi = _dev_mask(G, oracle_mod.random_mask(96, 64, 1))
+    mo = _dev_mask(G, oracle_mod.random_mask(160, 64, 2))
+    a = G.factgrass_compress(A, Gt, mi, mo, 512, 1, 9)
+    A2 = torch.cat([A, torch.randn_like(A)], dim=1).contiguous()
+    G2 = torch.cat([Gt, torch.zeros_like(Gt)], dim=1).contiguous()
+    b = G.factgrass_compress(A2, G2, mi, mo, 512, 1, 9)
+    assert torch.equal(a, b)
+
+
+def test_factgrass_errors_and_empty(G, W, oracle_mod):
+    cfg = _fact_cfg(W)
+    A, Gt = W.layer_io(cfg, 0, device="cuda")
+    mi = oracle_mod.random_mask(96, 24, 1)
+    mo = oracle_mod.random_mask(160, 40, 2)
+    # T = 0: zero output
+    o = torch.full((3, 97), 5.0, device="cuda")
+    G.factgrass_compress(A[:, :0].contiguous(), Gt[:, :0].contiguous(), _dev_mask(G, mi), _dev_mask(G, mo), 97, 1, 0, out=o)
+    assert torch.all(o == 0)
+    # fp32 inputs: unsupported
+    with pytest.raises(G.GrassError) as e:
+        G.factgrass_compress(A.float(), Gt.float(), _dev_mask(G, mi), _dev_mask(G, mo), 97, 1, 0)
+    assert e.value.code == 3
+    # an out-of-range mask index is skipped and flagged
+    bad = mo.copy()
+    bad[-1] = 4_000_000_000
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = G.factgrass_compress(A, Gt, _dev_mask(G, mi), _dev_mask(G, bad), 97, 1, 0, dev_status=st).cpu().numpy()
+    assert int(st.item()) & 1
+    G0 = Gt.clone()
+    G0[:, :, int(mo[-1])] = 0
+    ref, absum = oracle_mod.factgrass(W.bits_of(A), W.bits_of(G0), mi, mo, 97, 1, 0)
+    check_close(got, ref, absum, TOL_BF16, cfg.T + 64, eps=EPS_TC, what="bad factor index skipped")
+
+
+# ------------------------------------------------------------------ grouped
+
+def _group(G, W, oracle_mod, cfg, layer_ids, offsets=None):
+    layers, refs = [], []
+    off = 0
+    for n, l in enumerate(layer_ids):
+        lay = cfg.layers[l]
+        A, Gt = W.layer_io(cfg, l, device="cuda")
+        s_in, s_out = W.layer_mask_seeds(cfg, l)
+        mi = oracle_mod.random_mask(lay.d_in, cfg.kin, s_in)
+        mo = oracle_mod.random_mask(lay.d_out, cfg.kout, s_out)
+        o = off if offsets is None else offsets[n]
+        layers.append(dict(A=A, G=Gt, mask_in=_dev_mask(G, mi), mask_out=_dev_mask(G, mo), k=cfg.k, s=cfg.s,
+                           seed=W.layer_hash_seed(cfg, l), out_offset=o))
+        refs.append((o, mi, mo, W.layer_hash_seed(cfg, l), A, Gt))
+        off += cfg.k
+    return layers, refs
+
+
+def test_factgrass_grouped_parity(G, W, oracle_mod):
+    cfg = dataclasses.replace(W.CONFIG4, B=3, T=96, layers=W.CONFIG4.layers[:8])
+    ids = list(range(8))
+    layers, refs = _group(G, W, oracle_mod, cfg, ids)
+    group = G.GroupedLayers(layers)
+    ld = cfg.k * len(ids) + 5
+    out = torch.full((cfg.B, ld), 3.0, device="cuda")
+    ws = torch.empty(G.factgrass_grouped_workspace_bytes(len(ids)), dtype=torch.uint8, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    G.factgrass_compress_grouped(group, out, ws, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    host = out.cpu().numpy()
+    assert np.all(host[:, cfg.k * len(ids):] == 3.0)            # columns outside every layer's range untouched
+    for (o, mi, mo, seed, A, Gt) in refs:
+        ref, absum = oracle_mod.factgrass(W.bits_of(A), W.bits_of(Gt), mi, mo, cfg.k, cfg.s, seed)
+        check_close(host[:, o:o + cfg.k], ref, absum, TOL_BF16, cfg.T + 64, eps=EPS_TC, what=f"grouped off={o}")
+        single = G.factgrass_compress(A, Gt, _dev_mask(G, mi), _dev_mask(G, mo), cfg.k, cfg.s, seed).cpu().numpy()
+        check_close(single, ref, absum, TOL_BF16, cfg.T + 64, eps=EPS_TC, what="single")
+
+
+def test_factgrass_grouped_mixed_layers(G, W, oracle_mod):
+    """Layers of one call may differ in d_in/d_out, mask sizes, k, s and seed."""
+    B, T = 2, 50
+    specs = [(96, 160, 24, 40, 97, 1), (200, 64, 64, 64, 1024, 1), (768, 3072, 100, 130, 300, 2)]
+    layers, refs, off = [], [], 0
+    for n, (d_in, d_out, kin, kout, k, s) in enumerate(specs):
+        cfg = _fact_cfg(W, layers=(W.LinearLayer("x", d_in, d_out),), B=B, T=T, kin=kin, kout=kout, k=k, s=s,
+                        data_seed=100 + n)
+        A, Gt = W.layer_io(cfg, 0, device="cuda")
+        mi = oracle_mod.random_mask(d_in, kin, n)
+        mo = oracle_mod.random_mask(d_out, kout, n + 50)
+        layers.append(dict(A=A, G=Gt, mask_in=_dev_mask(G, mi), mask_out=_dev_mask(G, mo), k=k, s=s, seed=n * 3,
+                           out_offset=off))
+        refs.append((off, k, s, n * 3, mi, mo, A, Gt))
+        off += k + 3
+    out = torch.zeros(B, off, device="cuda")
+    ws = torch.empty(G.factgrass_grouped_workspace_bytes(len(specs)), dtype=torch.uint8, device="cuda")
+    G.factgrass_compress_grouped(G.GroupedLayers(layers), out, ws)
+    host = out.cpu().numpy()
+    for (o, k, s, seed, mi, mo, A, Gt) in refs:
+        ref, absum = oracle_mod.factgrass(W.bits_of(A), W.bits_of(Gt), mi, mo, k, s, seed)
+        check_close(host[:, o:o + k], ref, absum, TOL_BF16, T + 64, eps=EPS_TC, what=f"mixed off={o}")
+
+
+# ------------------------------------------------------------------ grass_score
+
+@pytest.mark.parametrize("N,M,D", [(300, 70, 257), (128, 128, 64), (1, 1, 1), (513, 256, 4096), (5, 3, 10)])
+def test_grass_score_parity(G, W, oracle_mod, N, M, D):
+    tr, te = W.score_vectors(N, M, D, 31, device="cuda")
+    sc = G.grass_score(tr, te).cpu().numpy()
+    ref, absum = oracle_mod.score(tr.cpu().numpy(), te.cpu().numpy())
+    check_close(sc, ref, absum, TOL_F32, D + 8, what=f"score {N}x{M}x{D}")
+
+
+def test_grass_score_strided_and_compressed_inputs(G, W, oracle_mod):
+    """Scores of actual compressed gradients; train rows taken from a wider matrix."""
+    g = W.dense_gradients(40, 30_000, 0.7, "normal", 1.0, 9, device="cuda")
+    idx = _dev_mask(G, oracle_mod.random_mask(30_000, 6_000, 0))
+    comp = G.grass_compress(g, idx, 510, 1, 4)
+    wide = torch.zeros(40, 520, device="cuda")
+    wide[:, :510] = comp
+    tr, te = wide[:30, :510], comp[30:]
+    sc = G.grass_score(tr, te).cpu().numpy()
+    ref, absum = oracle_mod.score(np.ascontiguousarray(tr.cpu().numpy()), np.ascontiguousarray(te.cpu().numpy()))
+    check_close(sc, ref, absum, TOL_F32, 520, what="score of compressed")
