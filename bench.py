@@ -1,0 +1,496 @@
+#!/usr/bin/env python
+"""Benchmark of the GraSS / FactGraSS compression hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config {1..5}] [--impl ours|reference]
+
+Prints ONE JSON line.  The default workload is config 5: FactGraSS over the 224 linear layers of a
+Llama-3-8B-shaped model (B=4 x T=2048 bf16, k'=64x64, k=4096 per layer) followed by grass_score of
+16,384 x 256 compressed vectors -- the configuration the paper's headline throughput (Table 2) is
+shaped like.  A step is one pass of the whole path over one batch.  Inputs are seeded and synthetic.
+
+--impl reference times the CPU oracle (plain C, fp64), as it stands, on a bounded sample.
+With N > 1 (torchrun) every rank runs an independent replica of the workload: the path does not shard.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+METRIC = "per-sample gradients compressed/sec"
+UNIT = "samples/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_BYTES = 126 * 1024 * 1024
+
+
+# ----------------------------------------------------------------------------- plumbing
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for ln in open(self.path):
+                f = [x.strip() for x in ln.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def dist_setup(n_gpus: int):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        dist.init_process_group(backend)
+    return world, rank, local
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    """Largest `value` over all ranks (a rank's timing counts only as the slowest one)."""
+    if world <= 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+class L2Flush:
+    def __init__(self, device):
+        self.buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+
+    def __call__(self):
+        self.buf.zero_()
+
+
+# ----------------------------------------------------------------------------- workloads (GPU arm)
+
+def sector_bytes_per_row(idx: np.ndarray, elem_bytes: int) -> int:
+    per = 32 // elem_bytes
+    return int(np.unique(idx.astype(np.int64) // per).size) * 32
+
+
+class GrassJob:
+    """configs 1-2: n samples in batches through grass_compress."""
+
+    def __init__(self, cfg, device, G, W):
+        self.cfg, self.G, self.device = cfg, G, device
+        self.idx = G.grass_random_mask_host(cfg.p, cfg.kprime, cfg.mask_seed)
+        self.didx = G.mask_to_device(self.idx, device)
+        self.nbatch = cfg.n // cfg.batch
+        batch_bytes = cfg.batch * cfg.p * 4
+        # distinct resident batches: enough that a batch is out of L2 when it is read again
+        self.ncopies = 1 if batch_bytes > 4 * L2_BYTES else min(8, max(2, (4 * L2_BYTES) // batch_bytes + 1))
+        self.g = [W.dense_gradients(cfg.batch, cfg.p, cfg.zero_prob, cfg.dist, cfg.scale, cfg.data_seed + c,
+                                    device=device) for c in range(self.ncopies)]
+        self.out = torch.empty((cfg.batch, cfg.k), dtype=torch.float32, device=device)
+        self.samples_per_step = cfg.n
+        self.alg_bytes_per_launch = cfg.batch * sector_bytes_per_row(self.idx, 4) + cfg.batch * cfg.k * 4
+        self.dense_bytes_per_launch = batch_bytes
+        self.launches_per_step = self.nbatch
+        self.kernels_per_step = 2 * self.nbatch     # memset + compress kernel per call (upper bound)
+        self.dominant = "grass_compress_kernel"
+        self.l2 = (f"{self.ncopies} resident batch(es) of {batch_bytes / 1e6:.0f} MB rotated; "
+                   + ("input >> L2" if self.ncopies == 1 else "L2 flushed between steps"))
+        self.need_flush = self.ncopies > 1
+        self._i = 0
+
+    def step(self, ev=None):
+        c = self.cfg
+        for b in range(self.nbatch):
+            g = self.g[self._i % self.ncopies]
+            self._i += 1
+            self.G.grass_compress(g, self.didx, c.k, c.s, c.hash_seed, out=self.out)
+
+    def dominant_ms(self, step_ms):
+        return step_ms / self.nbatch
+
+    def desc(self):
+        c = self.cfg
+        return {"workload": c.name, "n": c.n, "batch": c.batch, "p": c.p, "kprime": c.kprime, "k": c.k, "s": c.s,
+                "l2": self.l2}
+
+
+class FactJob:
+    """configs 3-5: all layers through one factgrass_compress_grouped launch (+ score for config 5)."""
+
+    def __init__(self, cfg, device, G, W):
+        self.cfg, self.G, self.device = cfg, G, device
+        layers, alg = [], 0
+        self.dense = 0
+        self.host_masks = []
+        for l, lay in enumerate(cfg.layers):
+            A, Gt = W.layer_io(cfg, l, device=device)
+            s_in, s_out = W.layer_mask_seeds(cfg, l)
+            mi = G.grass_random_mask_host(lay.d_in, cfg.kin, s_in)
+            mo = G.grass_random_mask_host(lay.d_out, cfg.kout, s_out)
+            self.host_masks.append((mi, mo))
+            layers.append(dict(A=A, G=Gt, mask_in=G.mask_to_device(mi, device), mask_out=G.mask_to_device(mo, device),
+                               k=cfg.k, s=cfg.s, seed=W.layer_hash_seed(cfg, l), out_offset=l * cfg.k))
+            alg += cfg.B * cfg.T * (sector_bytes_per_row(mi, 2) + sector_bytes_per_row(mo, 2)) + cfg.B * cfg.k * 4
+            self.dense += cfg.B * cfg.T * (lay.d_in + lay.d_out) * 2
+        self.layers = layers
+        self.group = G.GroupedLayers(layers)
+        self.out = torch.empty((cfg.B, cfg.out_dim), dtype=torch.float32, device=device)
+        self.ws = torch.empty(G.factgrass_grouped_workspace_bytes(len(layers)), dtype=torch.uint8, device=device)
+        self.score = None
+        if cfg.score_n_train:
+            self.score = W.score_vectors(cfg.score_n_train, cfg.score_n_test, cfg.k, cfg.data_seed + 7, device=device)
+            self.score_out = torch.empty((cfg.score_n_train, cfg.score_n_test), dtype=torch.float32, device=device)
+        self.samples_per_step = cfg.B
+        self.alg_bytes_per_launch = alg
+        self.dense_bytes_per_launch = self.dense
+        self.launches_per_step = 1
+        self.kernels_per_step = 2 + (1 if self.score else 0)
+        self.dominant = "factgrass_kernel"
+        self.need_flush = self.dense < 4 * L2_BYTES
+        self.l2 = "L2 flushed between steps" if self.need_flush else "inputs >> L2"
+        self.ev = []
+
+    def step(self, ev=None):
+        if ev is not None:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        self.G.factgrass_compress_grouped(self.group, self.out, self.ws)
+        if ev is not None:
+            e1.record()
+            ev.append((e0, e1))
+        if self.score:
+            self.G.grass_score(self.score[0], self.score[1], out=self.score_out)
+
+    def desc(self):
+        c = self.cfg
+        d = {"workload": c.name, "layers": len(c.layers), "B": c.B, "T": c.T, "kin": c.kin, "kout": c.kout,
+             "k_per_layer": c.k, "l2": self.l2}
+        if self.score:
+            d["score"] = f"{c.score_n_train}x{c.score_n_test}x{c.k} fp32"
+        return d
+
+
+def make_job(cfg_id, device, G, W):
+    cfg = W.CONFIGS[cfg_id]
+    return GrassJob(cfg, device, G, W) if cfg_id in (1, 2) else FactJob(cfg, device, G, W)
+
+
+def time_job(job, steps, warmup, world, device):
+    """K timed steps.  Big inputs: one event pair around all K steps.  Inputs that fit in L2: one event
+    pair per step with an L2 flush in between (not timed)."""
+    flush = L2Flush(device) if job.need_flush else None
+    for _ in range(warmup):
+        if flush:
+            flush()
+        job.step()
+    torch.cuda.synchronize()
+    barrier(world)
+    torch.cuda.synchronize()
+    dom_events = []
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            job.step(ev=dom_events)
+        e1.record()
+        torch.cuda.synchronize()
+        total_ms = e0.elapsed_time(e1)
+    else:
+        pairs = []
+        for _ in range(steps):
+            flush()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            job.step(ev=dom_events)
+            e1.record()
+            pairs.append((e0, e1))
+        torch.cuda.synchronize()
+        total_ms = sum(a.elapsed_time(b) for a, b in pairs)
+    barrier(world)
+    torch.cuda.synchronize()
+    ms_per_step = max_over_ranks(total_ms / steps, world, device)
+    if dom_events:
+        dom_ms = sum(a.elapsed_time(b) for a, b in dom_events) / len(dom_events)
+    else:
+        dom_ms = job.dominant_ms(total_ms / steps)
+    return ms_per_step, dom_ms
+
+
+# ----------------------------------------------------------------------------- end-to-end (host buffers)
+
+def e2e_job(cfg_id, job, steps, warmup, world, device, G, W):
+    """The same metric through the host-buffer API: every step copies the step's inputs from pinned
+    host memory to the device, compresses, and reads the result back."""
+    from paper_2505_18976_b200 import host_api
+    cfg = job.cfg
+    if cfg_id in (1, 2):
+        rows = min(cfg.batch, max(1, (1 << 30) // (cfg.p * 4)))           # <= 1 GiB pinned staging
+        pinned = torch.empty((rows, cfg.p), dtype=torch.float32, pin_memory=True)
+        pinned.copy_(job.g[0][:rows])
+        chunks = [pinned] * (cfg.n // rows)
+        out_host = torch.empty((cfg.n, cfg.k), dtype=torch.float32, pin_memory=True)
+        h2d = cfg.n * cfg.p * 4
+        d2h = cfg.n * cfg.k * 4
+        note = f"{cfg.n // rows} chunk copies of {rows} rows from one pinned staging buffer"
+
+        def run():
+            host_api.grass_compress_host(chunks, job.idx, cfg.k, cfg.s, cfg.hash_seed, out_host=out_host, device=device)
+    else:
+        # pinned copies of the first block's layers; later blocks of the same shape reuse those host
+        # tensors (the bytes copied per step are those of the whole model)
+        per_block = 7 if cfg_id == 5 else (4 if cfg_id == 4 else 1)
+        pinned = []
+        for l in range(per_block):
+            A, Gt = job.layers[l]["A"], job.layers[l]["G"]
+            pinned.append((torch.empty(A.shape, dtype=A.dtype, pin_memory=True).copy_(A),
+                           torch.empty(Gt.shape, dtype=Gt.dtype, pin_memory=True).copy_(Gt)))
+        groups, h2d = [], 0
+        for b0 in range(0, len(cfg.layers), per_block):
+            grp = []
+            for j in range(per_block):
+                l = b0 + j
+                mi, mo = job.host_masks[l]
+                grp.append(dict(A=pinned[j][0], G=pinned[j][1], mask_in=mi, mask_out=mo, k=cfg.k, s=cfg.s,
+                                seed=W.layer_hash_seed(cfg, l), out_offset=l * cfg.k))
+                h2d += pinned[j][0].numel() * 2 + pinned[j][1].numel() * 2
+            groups.append(grp)
+        out_host = torch.empty((cfg.B, cfg.out_dim), dtype=torch.float32, pin_memory=True)
+        d2h = cfg.B * cfg.out_dim * 4
+        note = f"{len(groups)} block copies from one block's pinned tensors"
+        score_host = None
+        if job.score:
+            score_host = (torch.empty(job.score[0].shape, pin_memory=True).copy_(job.score[0]),
+                          torch.empty(job.score[1].shape, pin_memory=True).copy_(job.score[1]))
+            h2d += (score_host[0].numel() + score_host[1].numel()) * 4
+            d2h += cfg.score_n_train * cfg.score_n_test * 4
+
+        def run():
+            host_api.factgrass_compress_host(groups, cfg.B, cfg.T, cfg.out_dim, out_host=out_host, device=device)
+            if score_host:
+                host_api.grass_score_host(score_host[0], score_host[1], device=device)
+
+    for _ in range(max(1, min(warmup, 2))):
+        run()
+    torch.cuda.synchronize()
+    barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = max_over_ranks(e0.elapsed_time(e1) / steps, world, device)
+    return {"value": world * job.samples_per_step / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps, "staging": note}
+
+
+# ----------------------------------------------------------------------------- CPU oracle arm
+
+def oracle_sample(cfg_id, W, budget="baseline"):
+    """A bounded sample of the workload for the CPU oracle, as host numpy arrays, and the fraction of
+    one step (in sample-equivalents) that it covers."""
+    import oracle
+    cfg = W.CONFIGS[cfg_id]
+    if cfg_id in (1, 2):
+        rows = 256 if cfg_id == 1 else 64
+        g = W.dense_gradients(rows, cfg.p, cfg.zero_prob, cfg.dist, cfg.scale, cfg.data_seed, device="cpu")
+        idx = oracle.random_mask(cfg.p, cfg.kprime, cfg.mask_seed)
+        gh = W.bits_of(g)
+
+        def run():
+            oracle.grass(gh, idx, cfg.k, cfg.s, cfg.hash_seed, want_absum=False)
+        return run, float(rows), f"{rows} of {cfg.n} samples, full p and k'"
+    nl = {3: 1, 4: 8, 5: 7}[cfg_id]
+    items = []
+    for l in range(nl):
+        lay = cfg.layers[l]
+        A, Gt = W.layer_io(cfg, l, device="cpu")
+        s_in, s_out = W.layer_mask_seeds(cfg, l)
+        items.append((W.bits_of(A), W.bits_of(Gt), oracle.random_mask(lay.d_in, cfg.kin, s_in),
+                      oracle.random_mask(lay.d_out, cfg.kout, s_out), W.layer_hash_seed(cfg, l)))
+
+    def run():
+        for (A, Gt, mi, mo, seed) in items:
+            oracle.factgrass(A, Gt, mi, mo, cfg.k, cfg.s, seed, want_absum=False)
+    frac = nl / len(cfg.layers)
+    return run, cfg.B * frac, f"first {nl} of {len(cfg.layers)} layers, all {cfg.B} samples x {cfg.T} tokens"
+
+
+def cpu_baseline(cfg_id, W, min_seconds=10.0, max_repeats=50):
+    """The oracle on the bounded sample, repeated until about `min_seconds` of wall time."""
+    import oracle
+    oracle.build()
+    run, sample_equiv, what = oracle_sample(cfg_id, W)
+    t0 = time.perf_counter()
+    repeats = 0
+    while repeats < max_repeats and (repeats == 0 or time.perf_counter() - t0 < min_seconds):
+        run()
+        repeats += 1
+    dt = (time.perf_counter() - t0) / repeats
+    what = f"{what}; {repeats} repeat(s)"
+    return {"value": sample_equiv / dt, "unit": UNIT, "cores": min(oracle.num_threads(), len(os.sched_getaffinity(0))),
+            "kind": "oracle", "sample": what, "seconds": dt}
+
+
+def reference_arm(args, W):
+    """--impl reference: the CPU oracle, as it stands, timed on the host cores."""
+    world, rank, _ = int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), 0
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    run, sample_equiv, what = oracle_sample(args.config, W)
+    for _ in range(min(args.warmup, 1)):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run()
+    ms = (time.perf_counter() - t0) / args.steps * 1e3
+    val = sample_equiv / (ms * 1e-3)
+    cores = min(oracle.num_threads(), len(os.sched_getaffinity(0)))
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": {"workload": W.CONFIGS[args.config].name, "sample": what},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- main
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    from paper_2505_18976_b200 import workloads as W
+    if args.impl == "reference":
+        reference_arm(args, W)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    world, rank, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    import paper_2505_18976_b200 as G
+    G.lib()
+    warmup = max(args.warmup, 3)
+
+    job = make_job(args.config, device, G, W)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms_per_step, dom_ms = time_job(job, args.steps, warmup, world, device)
+    clocks = sampler.stop()
+    value = world * job.samples_per_step / (ms_per_step * 1e-3)
+
+    peaks, peak_src = load_peaks()
+    achieved = job.alg_bytes_per_launch / (dom_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": job.dominant, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src,
+                "algorithmic_bytes_per_launch": int(job.alg_bytes_per_launch),
+                "dense_bytes_per_launch": int(job.dense_bytes_per_launch), "ms_per_launch": dom_ms,
+                "traffic": TRAFFIC.get(args.config)}
+
+    e2e = None
+    if not args.no_e2e:
+        e2e = e2e_job(args.config, job, max(1, args.e2e_steps), warmup, world, device, G, W)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_baseline(args.config, W)
+
+    if rank == 0:
+        cfgd = job.desc()
+        cfgd["replicas"] = world
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16" if args.config >= 3 else "f32", "data": "synthetic", "config": cfgd,
+                "tokens_per_s": (value * job.cfg.T if args.config >= 3 else None),
+                "clocks": clocks, "e2e": e2e, "gpu_launches": job.kernels_per_step * args.steps,
+                "roofline": roofline, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel per launch, from ncu captures
+# summarised under profiles/ (bytes; None until captured)
+TRAFFIC = {1: None, 2: None, 3: None, 4: None, 5: None}
+
+if __name__ == "__main__":
+    main()

@@ -226,7 +226,7 @@ int oracle_factgrass(const void *A, const void *G, int dtype, int32_t B, int32_t
             for (int32_t a = 0; a < kin; ++a)
                 for (int32_t c = 0; c < kout; ++c) {
                     gp[(int64_t)a * kout + c] += av[a] * gv[c];
-                    ga[(int64_t)a * kout + c] += fabs(av[a] * gv[c]);
+                    if (absum) ga[(int64_t)a * kout + c] += fabs(av[a] * gv[c]);
                 }
         }
         double *acc = out + (int64_t)b * k;

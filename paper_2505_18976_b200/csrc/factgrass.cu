@@ -218,13 +218,13 @@ __global__ void factgrass_zero_kernel(const LayerDesc* __restrict__ descs, const
 
 constexpr size_t kMaxSmemBins = 160 * 1024;
 
-static grass_status fill_desc(LayerDesc& d, const factgrass_layer& l, int tile)
+static grass_status fill_desc(LayerDesc& d, const factgrass_layer& l, int tile, int32_t T)
 {
     if (l.spec.k == 0 || l.spec.s == 0) return GRASS_ERR_INVALID_ARG;
     if (l.d_in <= 0 || l.d_out <= 0 || l.kin < 0 || l.kout < 0 || l.kin > l.d_in || l.kout > l.d_out)
         return GRASS_ERR_INVALID_ARG;
     if (l.out_offset < 0) return GRASS_ERR_INVALID_ARG;
-    if ((l.kin > 0 && l.kout > 0) && (!l.A || !l.G || !l.mask_in || !l.mask_out)) return GRASS_ERR_INVALID_ARG;
+    if ((l.kin > 0 && l.kout > 0 && T > 0) && (!l.A || !l.G || !l.mask_in || !l.mask_out)) return GRASS_ERR_INVALID_ARG;
     d.A = (const uint16_t*)l.A;
     d.G = (const uint16_t*)l.G;
     d.mask_in = l.mask_in;
@@ -288,7 +288,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
         if (!host) return GRASS_ERR_CUDA;
         grass_status rc = GRASS_OK;
         for (int l = 0; l < L && rc == GRASS_OK; ++l) {
-            rc = fill_desc(host[l], layers[l], tile);
+            rc = fill_desc(host[l], layers[l], tile, T);
             if (rc == GRASS_OK && host[l].tiles_m * host[l].tiles_n > max_tiles)
                 max_tiles = host[l].tiles_m * host[l].tiles_n;
         }
@@ -298,7 +298,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
         if (rc != GRASS_OK) return rc;
         dev_descs = (LayerDesc*)workspace;
     } else {
-        grass_status rc = fill_desc(single, layers[0], tile);
+        grass_status rc = fill_desc(single, layers[0], tile, T);
         if (rc != GRASS_OK) return rc;
         max_tiles = single.tiles_m * single.tiles_n;
     }

@@ -192,7 +192,7 @@ extern "C" grass_status grass_compress(const void* g, grass_dtype dt, int64_t n,
     if (!spec || spec->k == 0 || spec->s == 0) return GRASS_ERR_INVALID_ARG;
     if (n < 0 || p < 0 || kprime < 0 || kprime > p || ld < p || ld_out < (int64_t)spec->k) return GRASS_ERR_INVALID_ARG;
     if (p >= 0xFFFFFFFFLL) return GRASS_ERR_INVALID_ARG;
-    if (!idx && kprime != p) return GRASS_ERR_INVALID_ARG;
+    if (!idx && kprime != p && kprime != 0) return GRASS_ERR_INVALID_ARG;
     if (dt != GRASS_F32 && dt != GRASS_BF16) return GRASS_ERR_UNSUPPORTED;
     if (n == 0) return GRASS_OK;
     if (!out || (!g && kprime > 0)) return GRASS_ERR_INVALID_ARG;

@@ -260,7 +260,9 @@ def test_factgrass_padding_tokens_change_nothing(G, W, oracle_mod):
     A2 = torch.cat([A, torch.randn_like(A)], dim=1).contiguous()
     G2 = torch.cat([Gt, torch.zeros_like(Gt)], dim=1).contiguous()
     b = G.factgrass_compress(A2, G2, mi, mo, 512, 1, 9)
-    assert torch.equal(a, b)
+    # same sums, possibly split over different token chunks: equal up to fp32 rounding order
+    scale = float(a.abs().max())
+    assert float((a - b).abs().max()) <= 1e-5 * scale
 
 
 def test_factgrass_errors_and_empty(G, W, oracle_mod):
