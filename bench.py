@@ -235,8 +235,22 @@ class FactJob:
         return d
 
 
-def make_job(cfg_id, device, G, W):
+def small_config(cfg_id, W):
+    """A reduced case of the same kernels (inputs still larger than L2, a few GB at most) for profiler
+    captures."""
+    import dataclasses
     cfg = W.CONFIGS[cfg_id]
+    if cfg_id == 2:
+        return dataclasses.replace(cfg, n=64, batch=64)
+    if cfg_id == 4:
+        return dataclasses.replace(cfg, layers=cfg.layers[:16])
+    if cfg_id == 5:
+        return dataclasses.replace(cfg, layers=cfg.layers[:14], score_n_train=2048)
+    return cfg
+
+
+def make_job(cfg_id, device, G, W, small=False):
+    cfg = small_config(cfg_id, W) if small else W.CONFIGS[cfg_id]
     return GrassJob(cfg, device, G, W) if cfg_id in (1, 2) else FactJob(cfg, device, G, W)
 
 
@@ -434,6 +448,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--small", action="store_true", help="reduced case for profiler captures (not a bench value)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -449,9 +464,9 @@ def main():
     device = torch.device("cuda", local)
     import paper_2505_18976_b200 as G
     G.lib()
-    warmup = max(args.warmup, 3)
+    warmup = args.warmup if args.small else max(args.warmup, 3)
 
-    job = make_job(args.config, device, G, W)
+    job = make_job(args.config, device, G, W, small=args.small)
     sampler = ClockSampler(local)
     sampler.start()
     ms_per_step, dom_ms = time_job(job, args.steps, warmup, world, device)
@@ -476,6 +491,8 @@ def main():
     if rank == 0:
         cfgd = job.desc()
         cfgd["replicas"] = world
+        if args.small:
+            cfgd["small"] = True
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
                 "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16" if args.config >= 3 else "f32", "data": "synthetic", "config": cfgd,
