@@ -133,9 +133,11 @@ class L2Flush:
 
 # ----------------------------------------------------------------------------- workloads (GPU arm)
 
-def sector_bytes_per_row(idx: np.ndarray, elem_bytes: int) -> int:
-    per = 32 // elem_bytes
-    return int(np.unique(idx.astype(np.int64) // per).size) * 32
+def sector_bytes_per_row(idx: np.ndarray, elem_bytes: int, gran: int = 32) -> int:
+    """Bytes of one row that a gather of `idx` must move at `gran`-byte granularity (32 = L2 sector,
+    the algorithmic figure; 128 = the line the B200 memory system actually fetches)."""
+    per = gran // elem_bytes
+    return int(np.unique(idx.astype(np.int64) // per).size) * gran
 
 
 class GrassJob:
@@ -154,6 +156,7 @@ class GrassJob:
         self.out = torch.empty((cfg.batch, cfg.k), dtype=torch.float32, device=device)
         self.samples_per_step = cfg.n
         self.alg_bytes_per_launch = cfg.batch * sector_bytes_per_row(self.idx, 4) + cfg.batch * cfg.k * 4
+        self.line_bytes_per_launch = cfg.batch * sector_bytes_per_row(self.idx, 4, 128) + cfg.batch * cfg.k * 4
         self.dense_bytes_per_launch = batch_bytes
         self.launches_per_step = self.nbatch
         self.kernels_per_step = 2 * self.nbatch     # memset + compress kernel per call (upper bound)
@@ -184,7 +187,7 @@ class FactJob:
 
     def __init__(self, cfg, device, G, W):
         self.cfg, self.G, self.device = cfg, G, device
-        layers, alg = [], 0
+        layers, alg, line = [], 0, 0
         self.dense = 0
         self.host_masks = []
         for l, lay in enumerate(cfg.layers):
@@ -196,6 +199,7 @@ class FactJob:
             layers.append(dict(A=A, G=Gt, mask_in=G.mask_to_device(mi, device), mask_out=G.mask_to_device(mo, device),
                                k=cfg.k, s=cfg.s, seed=W.layer_hash_seed(cfg, l), out_offset=l * cfg.k))
             alg += cfg.B * cfg.T * (sector_bytes_per_row(mi, 2) + sector_bytes_per_row(mo, 2)) + cfg.B * cfg.k * 4
+            line += cfg.B * cfg.T * (sector_bytes_per_row(mi, 2, 128) + sector_bytes_per_row(mo, 2, 128)) + cfg.B * cfg.k * 4
             self.dense += cfg.B * cfg.T * (lay.d_in + lay.d_out) * 2
         self.layers = layers
         self.group = G.GroupedLayers(layers)
@@ -207,6 +211,7 @@ class FactJob:
             self.score_out = torch.empty((cfg.score_n_train, cfg.score_n_test), dtype=torch.float32, device=device)
         self.samples_per_step = cfg.B
         self.alg_bytes_per_launch = alg
+        self.line_bytes_per_launch = line
         self.dense_bytes_per_launch = self.dense
         self.launches_per_step = 1
         self.kernels_per_step = 2 + (1 if self.score else 0)
@@ -479,6 +484,9 @@ def main():
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": int(job.alg_bytes_per_launch),
                 "dense_bytes_per_launch": int(job.dense_bytes_per_launch), "ms_per_launch": dom_ms,
+                "line128_bytes_per_launch": int(job.line_bytes_per_launch),
+                "line128_achieved": job.line_bytes_per_launch / (dom_ms * 1e-3) / 1e9,
+                "line128_frac": job.line_bytes_per_launch / (dom_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                 "traffic": TRAFFIC.get(args.config)}
 
     e2e = None

@@ -15,7 +15,7 @@ import numpy as np
 import torch
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-SO_PATH = os.path.join(HERE, "libgrass_b200.so")
+SO_PATH = os.environ.get("GRASS_B200_LIB") or os.path.join(HERE, "libgrass_b200.so")
 
 GRASS_OK = 0
 STATUS = {0: "GRASS_OK", 1: "GRASS_ERR_INVALID_ARG", 2: "GRASS_ERR_BAD_MASK", 3: "GRASS_ERR_UNSUPPORTED",

@@ -22,7 +22,7 @@ def _stale() -> bool:
     if not os.path.exists(SO):
         return True
     t = os.path.getmtime(SO)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh", ".h"))]
     deps.append(os.path.join(os.path.dirname(HERE), "include", "grass.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
@@ -52,5 +52,17 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return SO
 
 
+def build_microbench() -> str:
+    """Compile the stand-alone DRAM fetch-granularity microbenchmark (not part of the library)."""
+    out = os.path.join(HERE, "_build", "fetch_granularity")
+    os.makedirs(os.path.dirname(out), exist_ok=True)
+    subprocess.check_call([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-o", out,
+                           os.path.join(CSRC, "microbench", "fetch_granularity.cu")])
+    return out
+
+
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--microbench" in sys.argv:
+        print(build_microbench())
+    else:
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

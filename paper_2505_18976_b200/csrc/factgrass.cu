@@ -110,12 +110,12 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
 #pragma unroll
         for (int i = 0; i < RA; ++i) {
             const int t = t0 + tokA + i * STEP_A;
-            ra[i] = (okA && t < t_end) ? __ldg(pA + (int64_t)t * d_in) : (uint16_t)0;
+            ra[i] = (okA && t < t_end) ? gather_u16(pA + (int64_t)t * d_in) : (uint16_t)0;
         }
 #pragma unroll
         for (int i = 0; i < RG; ++i) {
             const int t = t0 + tokG + i * STEP_G;
-            rg[i] = (okG && t < t_end) ? __ldg(pG + (int64_t)t * d_out) : (uint16_t)0;
+            rg[i] = (okG && t < t_end) ? gather_u16(pG + (int64_t)t * d_out) : (uint16_t)0;
         }
     };
     auto stash = [&](int buf) {

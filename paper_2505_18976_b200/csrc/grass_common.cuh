@@ -49,14 +49,54 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t b)
     return __uint_as_float((uint32_t)b << 16);
 }
 
+#ifndef GRASS_LD_MODE
+#define GRASS_LD_MODE 0
+#endif
+// gathered (scattered, read-once) loads of one element
+__device__ __forceinline__ uint32_t gather_u32(const uint32_t* p)
+{
+#if GRASS_LD_MODE == 0
+    return __ldg(p);
+#elif GRASS_LD_MODE == 1
+    return *p;
+#elif GRASS_LD_MODE == 2
+    return __ldcg(p);
+#elif GRASS_LD_MODE == 3
+    return __ldcs(p);
+#else
+    uint32_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.b32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+#endif
+}
+__device__ __forceinline__ uint16_t gather_u16(const uint16_t* p)
+{
+#if GRASS_LD_MODE == 0
+    return __ldg(p);
+#elif GRASS_LD_MODE == 1
+    return *p;
+#elif GRASS_LD_MODE == 2
+    return __ldcg(p);
+#elif GRASS_LD_MODE == 3
+    return __ldcs(p);
+#else
+    uint16_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.b16 %0, [%1];" : "=h"(v) : "l"(p));
+    return v;
+#endif
+}
+
 template <typename T> struct elem;
 template <> struct elem<float> {
-    static __device__ __forceinline__ float load(const float* p) { return __ldg(p); }
+    static __device__ __forceinline__ float load(const float* p)
+    {
+        return __uint_as_float(gather_u32(reinterpret_cast<const uint32_t*>(p)));
+    }
 };
 template <> struct elem<__nv_bfloat16> {
     static __device__ __forceinline__ float load(const __nv_bfloat16* p)
     {
-        return bf16_bits_to_float(__ldg(reinterpret_cast<const unsigned short*>(p)));
+        return bf16_bits_to_float(gather_u16(reinterpret_cast<const uint16_t*>(p)));
     }
 };
 
