@@ -118,6 +118,34 @@ grass_status factgrass_compress_grouped(const factgrass_layer* layers /*host*/, 
 size_t factgrass_grouped_workspace_bytes(int32_t L);
 
 /*
+ * factgrass_compress_grouped for callers that cannot hand over a device workspace.
+ * (An engineering variant: the paper has no counterpart to it.)
+ *
+ * Some callers are not in a position to allocate device memory at the moment they need to compress:
+ * a hook that runs in the middle of a backward pass under a framework whose memory pool already owns
+ * all of HBM, a serving or training loop that must not hit the implicit device synchronisation of
+ * cudaMalloc/cudaFree, or a plug-in whose host owns the allocator.  For them the layer descriptor
+ * table -- the only scratch the grouped kernels use -- is a fixed array inside the library image
+ * (22,528 bytes, resident on every GPU that loads the library until the process exits).  This call
+ * performs no cudaMalloc, cudaFree or other allocation, on the device or through any library.
+ *
+ *   Same arguments and results as factgrass_compress_grouped, minus workspace / workspace_bytes.
+ *   L may be at most FACTGRASS_STATIC_MAX_LAYERS (256); more returns GRASS_ERR_UNSUPPORTED with
+ *   nothing enqueued.  Split larger models over several calls (each on the same stream).
+ *   The first call on a device looks up the table's device address (once per device, with that device
+ *   current); make that first call outside any stream capture.
+ *   All calls on a device share the one table, and it keeps the previous call's descriptors until they
+ *   are overwritten: every call rewrites the L entries it uses before its kernels read them, nothing
+ *   else needs clearing.  Two calls whose GPU work can overlap (different streams, or different host
+ *   threads without ordering) race on the table; keep calls to this entry point on one stream, or
+ *   order them with events.
+ */
+#define FACTGRASS_STATIC_MAX_LAYERS 256
+grass_status factgrass_compress_grouped_static(const factgrass_layer* layers /*host*/, int32_t L, grass_dtype dt,
+                                               int32_t B, int32_t T, float* out, int64_t ld_out,
+                                               uint32_t* dev_status, void* stream);
+
+/*
  * Attribute-stage scores (Section 2.1): scores[i*ld_s + m] = <train[i, :], test[m, :]>.
  *   train N x D, test M x D, fp32 row-major with strides ld_train, ld_test >= D.
  *   scores N x M fp32 (train-major), row stride ld_s >= M.  Overwritten.  fp32 accumulation.

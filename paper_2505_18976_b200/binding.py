@@ -24,7 +24,7 @@ F32, BF16 = 0, 1
 DEV_BAD_INDEX, DEV_TIMEOUT = 1, 2
 
 EXPORTS = ("grass_compress", "factgrass_compress", "factgrass_compress_grouped",
-           "factgrass_grouped_workspace_bytes", "grass_score", "grass_sjlt_table", "grass_validate_mask",
+           "factgrass_grouped_workspace_bytes", "factgrass_compress_grouped_static", "grass_score", "grass_sjlt_table", "grass_validate_mask",
            "grass_random_mask_host", "grass_status_string")
 
 
@@ -67,6 +67,9 @@ def lib() -> ctypes.CDLL:
                                                  vp, ctypes.c_size_t, vp, vp]
         L.factgrass_grouped_workspace_bytes.restype = ctypes.c_size_t
         L.factgrass_grouped_workspace_bytes.argtypes = [i32]
+        L.factgrass_compress_grouped_static.restype = st
+        L.factgrass_compress_grouped_static.argtypes = [ctypes.POINTER(FactgrassLayer), i32, ctypes.c_int, i32, i32, vp,
+                                                        i64, vp, vp]
         L.grass_score.restype = st
         L.grass_score.argtypes = [vp, i64, i64, vp, i64, i64, i64, vp, i64, vp]
         L.grass_sjlt_table.restype = st
@@ -185,6 +188,23 @@ def factgrass_compress_grouped(group: GroupedLayers, out: torch.Tensor, workspac
                                             out.stride(0) if out.shape[0] > 1 else out.shape[1], _ptr(workspace),
                                             workspace.numel() * workspace.element_size(), _ptr(dev_status),
                                             _stream()), "factgrass_compress_grouped")
+    return out
+
+
+FACTGRASS_STATIC_MAX_LAYERS = 256   # FACTGRASS_STATIC_MAX_LAYERS in include/grass.h
+
+
+def factgrass_compress_grouped_static(group: GroupedLayers, out: torch.Tensor,
+                                      dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Grouped FactGraSS for callers that cannot allocate a device workspace (for example a hook running
+    while the framework's memory pool owns all of HBM): the descriptor table sits in a fixed array inside
+    the library, at most FACTGRASS_STATIC_MAX_LAYERS layers per call.  Calls share that table, so keep
+    them on one stream; the first call on a device should happen outside stream capture."""
+    _need_cuda(out, dev_status)
+    assert out.dtype == torch.float32 and out.stride(1) == 1
+    _check(lib().factgrass_compress_grouped_static(group.array, group.L, group.dtype, group.B, group.T, _ptr(out),
+                                                   out.stride(0) if out.shape[0] > 1 else out.shape[1],
+                                                   _ptr(dev_status), _stream()), "factgrass_compress_grouped_static")
     return out
 
 

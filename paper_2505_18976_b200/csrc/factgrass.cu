@@ -15,6 +15,7 @@
 
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 
 namespace grass {
 
@@ -380,5 +381,54 @@ extern "C" grass_status factgrass_compress_grouped(const factgrass_layer* layers
 {
     if (!workspace) return GRASS_ERR_INVALID_ARG;
     return grass::run_factgrass(layers, L, dt, B, T, out, ld_out, workspace, workspace_bytes, dev_status,
+                                (cudaStream_t)stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Grouped FactGraSS without a caller-provided workspace.
+//
+// The per-layer descriptor table of a grouped call is the only scratch memory the kernels need.
+// Here it lives in a fixed array that is part of the loaded library image on every GPU, so the call
+// needs no device allocation from anybody.  In host code the array's name is only a handle: the
+// device address is looked up once per device with cudaGetSymbolAddress and that pointer is what
+// the kernels receive.
+namespace grass {
+
+constexpr int kStaticMaxLayers = FACTGRASS_STATIC_MAX_LAYERS;
+static __device__ __align__(256) unsigned char g_static_layer_table[kStaticMaxLayers * sizeof(LayerDesc)];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mutex;
+static void* g_static_table_addr[kMaxDevices] = {nullptr};
+
+// Device address of the table on the current device; resolved on first use per device.
+static grass_status static_table_address(void** addr)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return GRASS_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_table_addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_layer_table) != cudaSuccess || !p) return GRASS_ERR_CUDA;
+        g_static_table_addr[dev] = p;
+    }
+    *addr = g_static_table_addr[dev];
+    return GRASS_OK;
+}
+
+}  // namespace grass
+
+extern "C" grass_status factgrass_compress_grouped_static(const factgrass_layer* layers, int32_t L, grass_dtype dt,
+                                                          int32_t B, int32_t T, float* out, int64_t ld_out,
+                                                          uint32_t* dev_status, void* stream)
+{
+    if (L < 0) return GRASS_ERR_INVALID_ARG;
+    if (L > grass::kStaticMaxLayers) return GRASS_ERR_UNSUPPORTED;  // table holds at most 256 layers
+    void* table = nullptr;
+    const grass_status rc = grass::static_table_address(&table);
+    if (rc != GRASS_OK) return rc;
+    return grass::run_factgrass(layers, L, dt, B, T, out, ld_out, table,
+                                (size_t)grass::kStaticMaxLayers * sizeof(grass::LayerDesc), dev_status,
                                 (cudaStream_t)stream);
 }
