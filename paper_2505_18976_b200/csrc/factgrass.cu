@@ -58,7 +58,7 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
 template <int TM, int TN>
 __global__ void __launch_bounds__(kFgThreads)
 factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ LayerDesc single, int32_t B,
-                 int32_t T, int32_t nchunks, int32_t chunk_len, float* __restrict__ out, int64_t ld_out,
+                 int32_t T, int32_t max_tiles, int32_t chunk_len, float* __restrict__ out, int64_t ld_out,
                  uint32_t* dev_status)
 {
     constexpr int PA = TM * 2 + 16;  // smem row pitch in bytes (tokens x masked columns, bf16)
@@ -77,8 +77,10 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     const LayerDesc& L = descs ? descs[blockIdx.z] : single;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.y;
-    const int chunk = blockIdx.x % nchunks;
-    const int tile = blockIdx.x / nchunks;
+    // block tiles of one token chunk are neighbours in launch order: the rows they share are read from
+    // HBM once and from L2 by the others
+    const int chunk = blockIdx.x / max_tiles;
+    const int tile = blockIdx.x % max_tiles;
     const int tm = tile % L.tiles_m, tn = tile / L.tiles_m;
     if (tn >= L.tiles_n) return;
     const int kin = L.kin, kout = L.kout;
@@ -273,7 +275,9 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
         if (layers[l].out_offset < 0 || layers[l].out_offset + (int64_t)layers[l].spec.k > ld_out)
             return GRASS_ERR_INVALID_ARG;
     }
-    const int tile = max_kk <= 64 ? 64 : 128;
+    // 64 x 64 block tiles (3 CTAs per SM); larger blocks are covered by several tiles whose shared rows
+    // come from L2.  The 128 x 128 variant (1 CTA per SM) is kept for comparison runs.
+    const int tile = fg_env_int("FACTGRASS_TILE", 64) == 128 && max_kk > 64 ? 128 : 64;
 
     const bool grouped = workspace != nullptr;
     if (!grouped && L != 1) return GRASS_ERR_INVALID_ARG;
@@ -317,11 +321,14 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
 
-    // token chunks: enough CTAs to fill the machine a few times over, but each chunk long enough
-    // that the fixed projection epilogue (tile*tile hashes) stays small beside the gather
+    // token chunks.  Every chunk pays a fixed projection epilogue (tile*tile hashes and a k-bin flush),
+    // so chunks are as long as the machine allows: when there are fewer work items than resident CTA
+    // slots the token sum is split just enough to fill one wave; otherwise just enough for ~8 waves
+    // so that the last, partial wave costs little.
     const int64_t base_items = (int64_t)L * B * max_tiles;
-    const int min_chunk = tile == 64 ? 128 : 64;
-    int64_t want = ((int64_t)sms * 8 + base_items - 1) / base_items;
+    const int64_t slots = (int64_t)sms * (tile == 64 ? 3 : 1);
+    const int min_chunk = 64;
+    int64_t want = base_items < slots ? slots / base_items : (8 * slots + base_items - 1) / base_items;
     int64_t max_chunks = (T + min_chunk - 1) / min_chunk;
     if (want > max_chunks) want = max_chunks;
     if (want < 1) want = 1;
@@ -340,7 +347,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
                 return GRASS_ERR_CUDA;
         }
-        kern<<<grid, kFgThreads, smem, st>>>(dev_descs, single, B, T, nchunks, chunk_len, out, ld_out, dev_status);
+        kern<<<grid, kFgThreads, smem, st>>>(dev_descs, single, B, T, max_tiles, chunk_len, out, ld_out, dev_status);
         return launch_status();
     };
     if (tile == 64) return launch(factgrass_kernel<64, 64>, (size_t)kTokTile * (2 * (64 * 2 + 16)));
