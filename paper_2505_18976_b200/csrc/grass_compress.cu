@@ -5,11 +5,16 @@
 // samples: S independent gathered loads per j are in flight together, consecutive lanes hold
 // consecutive (ascending) indices so the loads of a warp fall into the fewest 32-byte sectors.
 // Non-zero values are added into a per-sample k-bin accumulator in shared memory; exact zeros are
-// skipped (the input sparsity the paper's Section 3.1 builds on).  Bins are flushed with coalesced
-// stores, or with global reductions when the j range of a sample is split over several CTAs.
+// skipped (the input sparsity the paper's Section 3.1 builds on).  When the positions of a sample are
+// split over up to 8 CTAs, those CTAs form a thread-block cluster and add their bins through distributed
+// shared memory, each CTA storing one slice of the row: no zero-fill pass and no global atomics.  Wider
+// splits (few samples, very long masks) fall back to a zero-fill plus global reductions.
 #include "grass_common.cuh"
 
+#include <cooperative_groups.h>
 #include <cstdlib>
+
+namespace cg = cooperative_groups;
 
 namespace grass {
 
@@ -80,7 +85,24 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
     }
     if (bad && dev_status) atomicOr(dev_status, GRASS_DEV_BAD_INDEX);
 
-    if (use_smem) {
+    if (use_smem && accumulate == 2) {
+        // the gridDim.y CTAs that share these samples are one cluster: rank r sums slice r of every
+        // CTA's bins over distributed shared memory and stores it
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();
+        const uint32_t nr = cluster.num_blocks(), r = cluster.block_rank();
+        const uint32_t per = (k + nr - 1) / nr;
+        const uint32_t lo = r * per, hi = (lo + per) < k ? (lo + per) : k;
+        for (int si = 0; si < ns; ++si) {
+            float* dst = out + (i0 + si) * ld_out;
+            for (uint32_t i = lo + tid; i < hi; i += kThreads) {
+                float acc = 0.0f;
+                for (uint32_t q = 0; q < nr; ++q) acc += cluster.map_shared_rank(bins, q)[(uint32_t)si * k + i];
+                dst[i] = acc;
+            }
+        }
+        cluster.sync();  // nobody leaves while its bins may still be read
+    } else if (use_smem) {
         __syncthreads();
         for (int si = 0; si < ns; ++si) {
             float* dst = out + (i0 + si) * ld_out;
@@ -98,9 +120,10 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
 }
 
 struct CompressPlan {
-    int S;
-    int jsplit;
-    int use_smem;
+    int S;          // samples per CTA
+    int jsplit;     // CTAs that share one sample group (split of the masked positions)
+    int use_smem;   // k-bin accumulators fit in shared memory
+    int cluster;    // the jsplit CTAs are one thread-block cluster (DSMEM reduction)
 };
 
 static int env_int(const char* name, int dflt)
@@ -115,24 +138,34 @@ static CompressPlan plan_compress(int64_t n, int64_t kprime, uint32_t k, int sm_
     const size_t bin_bytes = (size_t)k * sizeof(float);
     const size_t smem_cap = 200 * 1024;
     pl.use_smem = bin_bytes <= smem_cap;
-    // samples per CTA: amortise the hash over S gathered loads, keep >= 3 CTAs per SM resident
-    int S = 4;
-    while (S > 1 && (bin_bytes * S > 64 * 1024 || (n + S - 1) / S < sm_count)) S >>= 1;
-    if (!pl.use_smem) S = 1;
-    S = env_int("GRASS_COMPRESS_S", S);
+    // One sample per CTA: the hash is a few dozen integer instructions per position, far below what the
+    // gathered loads leave idle, so sharing it between samples buys nothing and costs occupancy.
+    int S = env_int("GRASS_COMPRESS_S", 1);
     if (S != 1 && S != 2 && S != 4 && S != 8) S = 1;
     while (S > 1 && pl.use_smem && bin_bytes * S > smem_cap) S >>= 1;
+    if (!pl.use_smem) S = 1;
     pl.S = S;
+    const int U = S == 1 ? 8 : (S == 8 ? 2 : 4);
     const int64_t groups = (n + S - 1) / S;
-    const int64_t target = (int64_t)sm_count * 4;
-    int64_t js = (target + groups - 1) / (groups > 0 ? groups : 1);
-    // keep at least 8 positions per thread per CTA so the bin zero/flush is amortised
-    const int64_t max_js = kprime / (kThreads * 8) > 0 ? kprime / (kThreads * 8) : 1;
-    if (js > max_js) js = max_js;
-    if (js < 1) js = 1;
-    js = env_int("GRASS_COMPRESS_JSPLIT", (int)js);
+    // split positions until there are ~4 CTAs per SM, but keep one full round of loads per CTA
+    const int64_t max_js = kprime / ((int64_t)kThreads * U) > 0 ? kprime / ((int64_t)kThreads * U) : 1;
+    int64_t js = 1;
+    while (js < 8 && groups * js < (int64_t)sm_count * 4 && js * 2 <= max_js) js *= 2;
+    pl.cluster = 1;
+    if (groups * js < sm_count && js * 2 <= max_js) {
+        // very few samples: split wider than a cluster allows and reduce with global atomics
+        js = ((int64_t)sm_count * 2 + groups - 1) / groups;
+        if (js > max_js) js = max_js;
+        pl.cluster = 0;
+    }
+    const int forced = env_int("GRASS_COMPRESS_JSPLIT", 0);
+    if (forced > 0) {
+        js = forced;
+        pl.cluster = forced <= 8 && env_int("GRASS_COMPRESS_CLUSTER", 1) != 0;
+    }
     if (js < 1) js = 1;
     if (js > 65535) js = 65535;
+    if (js == 1 || !pl.use_smem) pl.cluster = 0;
     pl.jsplit = (int)js;
     return pl;
 }
@@ -144,18 +177,33 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
 {
     const int64_t groups = (n + S - 1) / S;
     const int64_t j_per_cta = (kprime + pl.jsplit - 1) / pl.jsplit;
-    const int accumulate = (pl.jsplit > 1 || !pl.use_smem) ? 1 : 0;
+    // 0: one CTA owns the row, plain stores; 1: global reductions into a zeroed row; 2: cluster reduction
+    const int accumulate = pl.cluster ? 2 : ((pl.jsplit > 1 || !pl.use_smem) ? 1 : 0);
     const size_t smem = pl.use_smem ? (size_t)S * sp.k * sizeof(float) : 0;
     const float scale = 1.0f / sqrtf((float)sp.s);
-    dim3 grid((unsigned)groups, (unsigned)pl.jsplit);
     auto launch = [&](auto kern) -> grass_status {
         if (smem > 48 * 1024) {
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return GRASS_ERR_CUDA;
         }
-        kern<<<grid, kThreads, smem, st>>>(g, n, p, ld, idx, kprime, sp.k, sp.s, sp.seed, scale, out, ld_out,
-                                           j_per_cta, accumulate, pl.use_smem, dev_status);
-        return launch_status();
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)groups, (unsigned)pl.jsplit, 1);
+        cfg.blockDim = dim3(kThreads, 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        if (pl.cluster) {
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 1;
+            attr[0].val.clusterDim.y = (unsigned)pl.jsplit;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+        }
+        const int use_smem = pl.use_smem;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, kern, g, n, p, ld, idx, kprime, sp.k, sp.s, sp.seed, scale, out,
+                                           ld_out, j_per_cta, accumulate, use_smem, dev_status);
+        return e == cudaSuccess ? launch_status() : GRASS_ERR_CUDA;
     };
     if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true>);
     return launch(grass_compress_kernel<T, S, U, false>);
@@ -170,7 +218,7 @@ static grass_status dispatch_compress(const T* g, int64_t n, int64_t p, int64_t 
     if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
     const CompressPlan pl = plan_compress(n, kprime, sp.k, sms);
-    if (pl.jsplit > 1 || !pl.use_smem) {
+    if (!pl.cluster && (pl.jsplit > 1 || !pl.use_smem)) {
         cudaError_t e = cudaMemset2DAsync(out, (size_t)ld_out * sizeof(float), 0, (size_t)sp.k * sizeof(float),
                                           (size_t)n, st);
         if (e != cudaSuccess) return GRASS_ERR_CUDA;
@@ -179,7 +227,7 @@ static grass_status dispatch_compress(const T* g, int64_t n, int64_t p, int64_t 
         case 8: return launch_compress<T, 8, 2>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
         case 4: return launch_compress<T, 4, 4>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
         case 2: return launch_compress<T, 2, 4>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
-        default: return launch_compress<T, 1, 4>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
+        default: return launch_compress<T, 1, 8>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
     }
 }
 

@@ -125,12 +125,15 @@ def test_grass_compress_student_t(G, W, oracle_mod):
     _grass_case(G, W, oracle_mod, 8, 1 << 18, 1 << 14, 4_096, zero_prob=0.7, dist="student_t3", scale=1e-2)
 
 
-@pytest.mark.parametrize("S,js", [(1, 1), (2, 3), (4, 7), (8, 2)])
-def test_grass_compress_launch_shapes(G, W, oracle_mod, monkeypatch, S, js):
-    """Every (samples per CTA, position split) plan gives the same answer."""
+@pytest.mark.parametrize("S,js,cluster", [(1, 1, 1), (2, 3, 0), (4, 7, 0), (8, 2, 1), (1, 2, 1), (1, 4, 1), (1, 8, 1),
+                                          (2, 4, 1), (1, 8, 0), (1, 20, 1)])
+def test_grass_compress_launch_shapes(G, W, oracle_mod, monkeypatch, S, js, cluster):
+    """Every plan (samples per CTA, position split, cluster or global-atomic reduction) gives the same answer."""
     monkeypatch.setenv("GRASS_COMPRESS_S", str(S))
     monkeypatch.setenv("GRASS_COMPRESS_JSPLIT", str(js))
+    monkeypatch.setenv("GRASS_COMPRESS_CLUSTER", str(cluster))
     _grass_case(G, W, oracle_mod, 11, 40_000, 9_000, 1_000)
+    _grass_case(G, W, oracle_mod, 5, 40_000, 9_000, 1_003, s=2)
 
 
 def test_grass_compress_special_values(G, oracle_mod):
