@@ -1,7 +1,12 @@
 // grass_score: scores[i, m] = <train[i, :], test[m, :]> (attribute stage, Section 2.1).
-// fp32 in, fp32 FMA accumulation.  128 x 128 output tile per CTA, 8 x 8 per thread, 16-deep
-// k tiles double-buffered through registers and shared memory.
+// The default path is the tensor-core kernel (split-bf16 products in tensor memory, see
+// grass_score_tc.cu).  This file holds the entry point and the plain fp32 FMA kernel (128 x 128 output
+// tile per CTA, 8 x 8 per thread, 16-deep k tiles double-buffered through registers and shared memory),
+// kept selectable with GRASS_SCORE_IMPL=ffma for comparison runs.
 #include "grass_common.cuh"
+
+#include <cstdlib>
+#include <cstring>
 
 namespace grass {
 
@@ -94,6 +99,9 @@ grass_score_kernel(const float* __restrict__ train, int64_t N, int64_t ld_train,
     }
 }
 
+grass_status launch_score_tc(const float* train, int64_t N, int64_t ld_train, const float* test, int64_t M,
+                             int64_t ld_test, int64_t D, float* scores, int64_t ld_s, cudaStream_t st);
+
 }  // namespace grass
 
 extern "C" grass_status grass_score(const float* train, int64_t N, int64_t ld_train, const float* test, int64_t M,
@@ -102,6 +110,9 @@ extern "C" grass_status grass_score(const float* train, int64_t N, int64_t ld_tr
     if (N < 0 || M < 0 || D < 0 || ld_train < D || ld_test < D || ld_s < M) return GRASS_ERR_INVALID_ARG;
     if (N == 0 || M == 0) return GRASS_OK;
     if (!scores || (D > 0 && (!train || !test))) return GRASS_ERR_INVALID_ARG;
+    const char* impl = std::getenv("GRASS_SCORE_IMPL");
+    if (!impl || std::strcmp(impl, "ffma") != 0)
+        return grass::launch_score_tc(train, N, ld_train, test, M, ld_test, D, scores, ld_s, (cudaStream_t)stream);
     const int64_t gx = (N + grass::SC_BM - 1) / grass::SC_BM, gy = (M + grass::SC_BN - 1) / grass::SC_BN;
     if (gx > 0x7FFFFFFFLL || gy > 65535) return GRASS_ERR_UNSUPPORTED;
     const int vec_ok = ((uintptr_t)train % 16 == 0) && ((uintptr_t)test % 16 == 0) && (ld_train % 4 == 0) &&
