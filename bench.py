@@ -515,7 +515,8 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel per launch, from ncu captures
 # summarised under profiles/ (bytes; None until captured)
-TRAFFIC = {1: None, 2: None, 3: None, 4: None, 5: None}
+TRAFFIC = {1: 65_797_632 + 326_400, 2: 8 * (425_576_704 + 3_593_984), 3: 124_362_496 + 4_034_048, 4: None,
+           5: 16 * (1_191_473_000 + 5_273_600)}
 
 if __name__ == "__main__":
     main()
