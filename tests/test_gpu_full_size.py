@@ -1,0 +1,165 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration the benchmark times.
+
+Every configuration is run exactly as ``bench.py`` runs it (same workload generators, same
+calls, whole batch / all layers in one launch).  Where the CPU oracle can do the whole output in
+seconds (configs 1 and 3) every element is compared; otherwise the outputs of a sample of rows
+or layers are recomputed by the oracle from the same bytes, and the rest is checked by
+properties that hold at any size (finite, untouched neighbours, mass that matches the input).
+"""
+import numpy as np
+import pytest
+import torch
+
+from parity import check_close, max_bin_load
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32, TOL_BF16 = 1e-4, 2e-2
+EPS_TC = 2.0 ** -23
+
+
+@pytest.fixture(scope="module")
+def G():
+    import paper_2505_18976_b200 as g
+    g.lib()
+    return g
+
+
+@pytest.fixture(scope="module")
+def W():
+    from paper_2505_18976_b200 import workloads
+    return workloads
+
+
+@pytest.fixture(autouse=True)
+def _release_memory():
+    yield
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+
+
+def test_config1_full_every_output(G, W, oracle_mod):
+    c = W.CONFIG1
+    g = W.dense_gradients(c.batch, c.p, c.zero_prob, c.dist, c.scale, c.data_seed, device="cuda")
+    idx = G.grass_random_mask_host(c.p, c.kprime, c.mask_seed)
+    assert np.array_equal(idx, oracle_mod.random_mask(c.p, c.kprime, c.mask_seed))
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = G.grass_compress(g, G.mask_to_device(idx), c.k, c.s, c.hash_seed, dev_status=st)
+    assert int(st.item()) == 0
+    ref, absum = oracle_mod.grass(W.bits_of(g), idx, c.k, c.s, c.hash_seed)
+    ob, _ = oracle_mod.sjlt_table(c.k, c.s, c.hash_seed, c.kprime)
+    check_close(out.cpu().numpy(), ref, absum, TOL_F32, max_bin_load(ob, c.k) + 16, what="config 1 full")
+
+
+def test_config2_full_batch_sampled_rows(G, W, oracle_mod):
+    """One batch of 512 x 4,194,304 fp32 (8.6 GB) through one call; the oracle recomputes 24 rows."""
+    c = W.CONFIG2
+    g = W.dense_gradients(c.batch, c.p, c.zero_prob, c.dist, c.scale, c.data_seed, device="cuda")
+    idx = G.grass_random_mask_host(c.p, c.kprime, c.mask_seed)
+    assert np.array_equal(idx, oracle_mod.random_mask(c.p, c.kprime, c.mask_seed))
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    wide = torch.full((c.batch, c.k + 3), 9.0, device="cuda")              # a strided output with a guard band
+    out = wide[:, :c.k]
+    G.grass_compress(g, G.mask_to_device(idx), c.k, c.s, c.hash_seed, out=out, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    rows = sorted(set([0, 1, 255, 256, 510, 511] + list(np.random.default_rng(2).integers(0, c.batch, 18))))
+    sample = g[rows].cpu().numpy()
+    ref, absum = oracle_mod.grass(sample, idx, c.k, c.s, c.hash_seed)
+    ob, _ = oracle_mod.sjlt_table(c.k, c.s, c.hash_seed, c.kprime)
+    host = out.cpu().numpy()
+    check_close(host[rows], ref, absum, TOL_F32, max_bin_load(ob, c.k) + 16, what="config 2 sampled rows")
+    # every row: finite, and the signed total of a row equals the signed total of its masked entries
+    assert np.isfinite(host).all()
+    didx = G.mask_to_device(idx).long()
+    sign = torch.from_numpy(oracle_mod.sjlt_table(c.k, c.s, c.hash_seed, c.kprime)[1].astype(np.float64)).cuda()
+    tot_ref = torch.zeros(c.batch, dtype=torch.float64, device="cuda")
+    mass = torch.zeros(c.batch, dtype=torch.float64, device="cuda")
+    for r0 in range(0, c.batch, 64):
+        gm = g[r0:r0 + 64].index_select(1, didx).double()
+        tot_ref[r0:r0 + 64] = (gm * sign).sum(1)
+        mass[r0:r0 + 64] = gm.abs().sum(1)
+    tot = out.double().sum(1)
+    assert torch.all((tot - tot_ref).abs() <= 1e-5 * mass)
+    assert torch.all(wide[:, c.k:] == 9.0)
+
+
+def test_config3_full_every_output(G, W, oracle_mod):
+    c = W.CONFIG3
+    lay = c.layers[0]
+    A, Gt = W.layer_io(c, 0, device="cuda")
+    s_in, s_out = W.layer_mask_seeds(c, 0)
+    mi = G.grass_random_mask_host(lay.d_in, c.kin, s_in)
+    mo = G.grass_random_mask_host(lay.d_out, c.kout, s_out)
+    seed = W.layer_hash_seed(c, 0)
+    layers = [dict(A=A, G=Gt, mask_in=G.mask_to_device(mi), mask_out=G.mask_to_device(mo), k=c.k, s=c.s, seed=seed,
+                   out_offset=0)]
+    out = torch.empty(c.B, c.k, device="cuda")
+    ws = torch.empty(G.factgrass_grouped_workspace_bytes(1), dtype=torch.uint8, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    G.factgrass_compress_grouped(G.GroupedLayers(layers), out, ws, dev_status=st)
+    assert int(st.item()) == 0
+    ref, absum = oracle_mod.factgrass(W.bits_of(A), W.bits_of(Gt), mi, mo, c.k, c.s, seed)
+    ob, _ = oracle_mod.sjlt_table(c.k, c.s, seed, c.kin * c.kout)
+    check_close(out.cpu().numpy(), ref, absum, TOL_BF16, c.T + max_bin_load(ob, c.k) + 64, eps=EPS_TC,
+                what="config 3 full")
+
+
+def _grouped_full(G, W, oracle_mod, c, sample_layers, what):
+    layers, keep = [], {}
+    for l, lay in enumerate(c.layers):
+        A, Gt = W.layer_io(c, l, device="cuda")
+        s_in, s_out = W.layer_mask_seeds(c, l)
+        mi = G.grass_random_mask_host(lay.d_in, c.kin, s_in)
+        mo = G.grass_random_mask_host(lay.d_out, c.kout, s_out)
+        layers.append(dict(A=A, G=Gt, mask_in=G.mask_to_device(mi), mask_out=G.mask_to_device(mo), k=c.k, s=c.s,
+                           seed=W.layer_hash_seed(c, l), out_offset=l * c.k))
+        if l in sample_layers:
+            keep[l] = (mi, mo)
+    out = torch.full((c.B, c.out_dim), float("nan"), device="cuda")
+    ws = torch.empty(G.factgrass_grouped_workspace_bytes(len(layers)), dtype=torch.uint8, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    G.factgrass_compress_grouped(G.GroupedLayers(layers), out, ws, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    host = out.cpu().numpy()
+    assert np.isfinite(host).all()                       # every layer's range was written
+    per_layer_mass = np.abs(host).reshape(c.B, len(c.layers), c.k).sum(2)
+    assert (per_layer_mass > 0).all()
+    for l in sorted(sample_layers):
+        mi, mo = keep[l]
+        seed = W.layer_hash_seed(c, l)
+        assert np.array_equal(mi, oracle_mod.random_mask(c.layers[l].d_in, c.kin, W.layer_mask_seeds(c, l)[0]))
+        ref, absum = oracle_mod.factgrass(W.bits_of(layers[l]["A"]), W.bits_of(layers[l]["G"]), mi, mo, c.k, c.s, seed)
+        ob, _ = oracle_mod.sjlt_table(c.k, c.s, seed, c.kin * c.kout)
+        check_close(host[:, l * c.k:(l + 1) * c.k], ref, absum, TOL_BF16, c.T + max_bin_load(ob, c.k) + 64,
+                    eps=EPS_TC, what=f"{what} layer {l} ({c.layers[l].name})")
+    return out
+
+
+def test_config4_full_all_layers_one_launch(G, W, oracle_mod):
+    """48 layers x 16 x 1,024 tokens in one grouped launch; the oracle recomputes 12 of the layers."""
+    _grouped_full(G, W, oracle_mod, W.CONFIG4, {0, 1, 2, 3, 9, 14, 20, 27, 33, 38, 46, 47}, "config 4")
+
+
+def test_config5_full_all_layers_one_launch_and_score(G, W, oracle_mod):
+    """224 layers x 4 x 2,048 tokens (42.9 GB resident) in one grouped launch; the oracle recomputes 10 layers,
+    one of every shape among them; then the full-size score with 256 sampled train rows."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 * 2 ** 30:
+        pytest.skip("needs about 50 GB of free device memory")
+    c = W.CONFIG5
+    _grouped_full(G, W, oracle_mod, c, {0, 1, 2, 3, 4, 5, 6, 108, 117, 223}, "config 5")
+    torch.cuda.empty_cache()
+    tr, te = W.score_vectors(c.score_n_train, c.score_n_test, c.k, c.data_seed + 7, device="cuda")
+    sc = G.grass_score(tr, te)
+    rows = sorted(set([0, 127, 128, 16_383] + list(np.random.default_rng(5).integers(0, c.score_n_train, 252))))
+    ref, absum = oracle_mod.score(tr[rows].cpu().numpy(), te.cpu().numpy())
+    check_close(sc[rows].cpu().numpy(), ref, absum, TOL_F32, c.k + 8, what="config 5 score, sampled train rows")
+    # all rows: Cauchy-Schwarz and the row sum <train_i, sum_m test_m>
+    assert torch.isfinite(sc).all()
+    bound = tr.double().norm(dim=1)[:, None] * te.double().norm(dim=1)[None, :]
+    assert torch.all(sc.double().abs() <= bound * (1 + 1e-6))
+    rowsum = tr.double() @ te.double().sum(0)
+    absrow = tr.double().abs() @ te.double().abs().sum(0)
+    assert torch.all((sc.double().sum(1) - rowsum).abs() <= 1e-5 * absrow)
