@@ -5,6 +5,7 @@
 // Every wait on an mbarrier is bounded and the kernel leaves with a flag set if one expires.
 #include <cstdio>
 #include <cstdint>
+#include <cstdlib>
 #include <cuda_runtime.h>
 #define CK(x) do{cudaError_t e=(x); if(e!=cudaSuccess){printf("err %s line %d\n", cudaGetErrorString(e), __LINE__); return 1;}}while(0)
 
@@ -68,6 +69,14 @@ __global__ void rd_bulk(const uint32_t* __restrict__ p, size_t n_reads, size_t s
 
 int main(int argc, char** argv)
 {
+    // optional argument: value for cudaLimitMaxL2FetchGranularity (32, 64 or 128), set before anything
+    // else touches the device; the value the driver reports back is printed
+    if (argc > 1) {
+        CK(cudaDeviceSetLimit(cudaLimitMaxL2FetchGranularity, (size_t)atoi(argv[1])));
+    }
+    size_t gran = 0;
+    CK(cudaDeviceGetLimit(&gran, cudaLimitMaxL2FetchGranularity));
+    printf("cudaLimitMaxL2FetchGranularity = %zu\n", gran);
     const size_t bytes = 2ull << 30;
     uint32_t *p, *out;
     CK(cudaMalloc(&p, bytes)); CK(cudaMemset(p, 1, bytes)); CK(cudaMalloc(&out, 64)); CK(cudaMemset(out, 0, 64));
