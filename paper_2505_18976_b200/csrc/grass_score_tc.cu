@@ -4,14 +4,14 @@
 // of the path.  fp32 inputs are split exactly into three bf16 pieces, x = hi + mid + lo (8 significant
 // bits each, by truncation), and the product is rebuilt from the six partial products whose weight is
 // at least 2^-16 of the leading one (hi*hi, hi*mid, mid*hi, mid*mid, hi*lo, lo*hi); what is dropped is
-// below 2^-23 of |x||y|, the size of one fp32 rounding.  All six accumulate into one fp32 tile in tensor
-// memory.
+// below 2^-23 of |x||y|, the size of one fp32 rounding.  hi*hi accumulates in one fp32 tile in tensor
+// memory and the five correction terms in a second one; the epilogue adds the two.
 //
 // One CTA owns a 128 x (<=256) output tile: 128 train rows (MMA M) by up to 256 test rows (MMA N).
-//   warps 0-7  producers: read fp32 rows from HBM (two stages of registers in flight), split, and write
-//              the bf16 pieces into shared memory in the tensor core's K-major core-matrix layout
-//              (8 rows x 16 bytes contiguous, no swizzle); afterwards they drain the accumulator;
-//   warp 8     one elected thread issues tcgen05.mma (M=128, N<=256, K=16) and commits stage-free and
+//   producer warps: read fp32 rows from HBM (the next k tile in registers while the current one is split),
+//              split, and write the bf16 pieces into shared memory in the tensor core's K-major layout with
+//              the 64-byte swizzle (64-byte rows; conflict-free 16-byte stores); then drain the accumulators;
+//   last warp  one elected thread issues tcgen05.mma (M=128, N<=256, K=16) and commits stage-free and
 //              accumulator-ready mbarriers.
 // Three 72 KB stages of 32 k-values each.  Every mbarrier wait is bounded: if one expires the CTA marks
 // its tile with NaN, still frees its tensor memory, and returns.
@@ -24,16 +24,26 @@ constexpr int BM = 128;            // train rows per CTA (MMA M)
 constexpr int BN = 256;            // test rows per CTA (MMA N, upper bound)
 constexpr int BK = 32;             // k values per stage
 constexpr int STAGES = 3;
-constexpr int PRODUCERS = 256;     // threads of warps 0-7
+#ifndef GRASS_SCORE_PRODUCERS
+#define GRASS_SCORE_PRODUCERS 512
+#endif
+#ifndef GRASS_SCORE_PREFETCH
+#define GRASS_SCORE_PREFETCH 1
+#endif
+constexpr int PRODUCERS = GRASS_SCORE_PRODUCERS;   // threads of the producer warps
+constexpr int PWARPS = PRODUCERS / 32;
+constexpr int PF = GRASS_SCORE_PREFETCH;           // k tiles of global loads in flight ahead of the one being split
+constexpr int RING = PF + 1;
 constexpr int THREADS = PRODUCERS + 32;
 constexpr int A_SPLIT_BYTES = BM * BK * 2;   // one bf16 piece of the train tile:  8 KB
 constexpr int B_SPLIT_BYTES = BN * BK * 2;   // one bf16 piece of the test tile:  16 KB
 constexpr int STAGE_BYTES = 3 * (A_SPLIT_BYTES + B_SPLIT_BYTES);   // 72 KB
 constexpr int CHUNKS = BK / 8;     // 16-byte chunks (8 bf16) per row per stage
 constexpr int TASKS = (BM + BN) * CHUNKS / PRODUCERS;   // (row, chunk) tasks per producer per stage = 6
-constexpr uint32_t LBO = 128;      // bytes between the core matrices of consecutive 8-value k chunks
-constexpr uint32_t SBO = CHUNKS * 128;   // bytes between consecutive 8-row groups
-constexpr uint32_t TMEM_COLS = 256;
+constexpr uint32_t ROW_BYTES = BK * 2;        // one row of a bf16 piece: 64 bytes = one 64-byte swizzle row
+constexpr uint32_t SBO = 8 * ROW_BYTES;       // bytes between consecutive 8-row groups (512)
+static_assert(ROW_BYTES == 64, "the shared-memory layout below is the 64-byte-swizzle K-major one");
+constexpr uint32_t TMEM_COLS = 512;   // two fp32 accumulators of BN columns each
 constexpr uint32_t SPIN_LIMIT = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -63,11 +73,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     return false;
 }
 
-// shared-memory matrix descriptor: K-major, no swizzle, version 1 (sm_100)
+// shared-memory matrix descriptor: K-major, 64-byte swizzle, version 1 (sm_100).  Rows are 64 bytes
+// apart, 8-row groups SBO apart; the 16-byte chunk c of row r sits at chunk position c ^ ((r >> 1) & 3)
+// (address bits [4,6) xor bits [7,9)).  The leading-dimension offset is not used by swizzled K-major
+// layouts (set to 16 bytes).
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr)
 {
-    return (uint64_t)((addr >> 4) & 0x3FFF) | ((uint64_t)(LBO >> 4) << 16) | ((uint64_t)(SBO >> 4) << 32) |
-           (1ull << 46);
+    return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(SBO >> 4) << 32) | (1ull << 46) |
+           (4ull << 61);
 }
 
 // instruction descriptor: D fp32, A and B bf16, both K-major, M x N
@@ -153,7 +166,7 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 8) {
+    if (warp == PWARPS) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                      "r"(TMEM_COLS)
                      : "memory");
@@ -165,11 +178,12 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
     const uint32_t tmem_d = tmem_base_slot;
     const uint32_t smem_base = smem_u32(smem);
 
-    if (warp < 8) {
+    if (warp < PWARPS) {
         // ---------------- producers ----------------
-        // task q of this thread: flat = tid + q * 256 -> row = flat / 4 over the 384 rows (train rows
-        // first), chunk = flat % 4
-        float raw[2][TASKS][8];
+        // task q of this thread: flat = tid + q * PRODUCERS -> row = flat / 4 over the 384 rows (train rows
+        // first), chunk = flat % 4: four lanes read one row's 128 contiguous bytes, and with the 64-byte
+        // swizzle the 16-byte stores of eight consecutive lanes (two rows) fill 128 contiguous bytes
+        float raw[RING][TASKS][8];
         auto fetch = [&](int64_t kt, float (&dst)[TASKS][8]) {
             const int64_t d0 = kt * BK;
 #pragma unroll
@@ -204,25 +218,30 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
                 split8(srcv[q], hi, mid, lo);
                 unsigned char* base = is_a ? st : st + 3 * A_SPLIT_BYTES;
                 const int piece = is_a ? A_SPLIT_BYTES : B_SPLIT_BYTES;
-                const int off = (r >> 3) * SBO + ch * LBO + (r & 7) * 16;
+                const int off = (r >> 3) * SBO + (r & 7) * ROW_BYTES + ((ch ^ ((r >> 1) & 3)) << 4);
                 *reinterpret_cast<uint4*>(base + off) = hi;
                 *reinterpret_cast<uint4*>(base + piece + off) = mid;
                 *reinterpret_cast<uint4*>(base + 2 * piece + off) = lo;
             }
         };
-        if (ktiles > 0) fetch(0, raw[0]);
+#pragma unroll
+        for (int q = 0; q < PF; ++q)
+            if (q < ktiles) fetch(q, raw[q]);
         bool ok = true;
-        for (int64_t kt = 0; kt < ktiles && ok; ++kt) {
-            const int s = (int)(kt % STAGES);
-            const uint32_t round = (uint32_t)(kt / STAGES);
-            if (kt + 1 < ktiles) {
-                if (kt & 1) fetch(kt + 1, raw[0]); else fetch(kt + 1, raw[1]);
+        for (int64_t kt0 = 0; kt0 < ktiles && ok; kt0 += RING) {
+#pragma unroll
+            for (int ph = 0; ph < RING; ++ph) {
+                const int64_t kt = kt0 + ph;
+                if (kt >= ktiles || !ok) break;
+                const int s = (int)(kt % STAGES);
+                const uint32_t round = (uint32_t)(kt / STAGES);
+                if (kt + PF < ktiles) fetch(kt + PF, raw[(ph + PF) % RING]);
+                if (round > 0) ok = mbar_wait(empty0 + 8 * s, (round - 1) & 1) && !abort_flag;
+                if (!ok) break;
+                stash(s, raw[ph]);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(full0 + 8 * s);
             }
-            if (round > 0) ok = mbar_wait(empty0 + 8 * s, (round - 1) & 1) && !abort_flag;
-            if (!ok) break;
-            if (kt & 1) stash(s, raw[1]); else stash(s, raw[0]);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            mbar_arrive(full0 + 8 * s);
         }
         if (!ok) abort_flag = 1;
 
@@ -231,15 +250,19 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
         if (!ok) abort_flag = 1;
         ok = __all_sync(0xFFFFFFFFu, ok);   // tensor-memory loads below are warp-collective
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        // warp w reads TMEM lanes 32*(w%4) .. +31 (= output rows); warps 0-3 take the even 32-column
-        // groups, warps 4-7 the odd ones
+        // warp w reads TMEM lanes 32*(w%4) .. +31 (= output rows); the PWARPS/4 warps that share a lane
+        // group take every (PWARPS/4)-th 32-column group
         const int lane_grp = warp & 3;
         const int64_t row = n0 + lane_grp * 32 + lane;
-        for (uint32_t c0 = (warp >> 2) * 32; c0 < n_mma; c0 += 64) {
+        for (uint32_t c0 = (warp >> 2) * 32; c0 < n_mma; c0 += 32 * (PWARPS / 4)) {
             uint32_t v[32];
             if (ok && ktiles > 0) {
+                uint32_t w[32];
                 tmem_ld32(tmem_d + ((uint32_t)(lane_grp * 32) << 16) + c0, v);
+                tmem_ld32(tmem_d + ((uint32_t)(lane_grp * 32) << 16) + BN + c0, w);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(w[e]));
             } else {
 #pragma unroll
                 for (int e = 0; e < 32; ++e) v[e] = (ktiles > 0) ? 0x7FC00000u : 0u;   // NaN marks an aborted tile
@@ -268,15 +291,18 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t a0 = smem_base + s * STAGE_BYTES, b0 = a0 + 3 * A_SPLIT_BYTES;
-            // (piece of A, piece of B): 0 = hi, 1 = mid, 2 = lo; small terms first
-            const int pa[6] = {2, 0, 1, 1, 0, 0}, pb[6] = {0, 2, 1, 0, 1, 0};
+            // (piece of A, piece of B): 0 = hi, 1 = mid, 2 = lo.  hi*hi goes to the first accumulator, the
+            // five correction terms (2^-8 and 2^-16 of it) to the second: the tensor core truncates after
+            // every accumulation, so the large sum should see as few of them as possible
+            const int pa[6] = {0, 2, 0, 1, 1, 0}, pb[6] = {0, 0, 2, 1, 0, 1};
 #pragma unroll
             for (int t = 0; t < 6; ++t) {
 #pragma unroll
                 for (int ks = 0; ks < BK / 16; ++ks) {
-                    const uint64_t ad = make_smem_desc(a0 + pa[t] * A_SPLIT_BYTES + ks * 2 * LBO);
-                    const uint64_t bd = make_smem_desc(b0 + pb[t] * B_SPLIT_BYTES + ks * 2 * LBO);
-                    umma_bf16(tmem_d, ad, bd, idesc, (kt > 0 || t > 0 || ks > 0) ? 1u : 0u);
+                    const uint64_t ad = make_smem_desc(a0 + pa[t] * A_SPLIT_BYTES + ks * 32);   // 16 k values on
+                    const uint64_t bd = make_smem_desc(b0 + pb[t] * B_SPLIT_BYTES + ks * 32);
+                    const uint32_t acc_on = (kt > 0 || ks > 0 || t > 1) ? 1u : 0u;
+                    umma_bf16(t == 0 ? tmem_d : tmem_d + BN, ad, bd, idesc, acc_on);
                 }
             }
             umma_commit(empty0 + 8 * s);   // stage s may be overwritten once these MMAs have read it
@@ -287,7 +313,7 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == 8) {
+    if (warp == PWARPS) {
         __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(TMEM_COLS) : "memory");
     }
