@@ -56,6 +56,9 @@ def lib() -> ctypes.CDLL:
         L.oracle_factgrass.restype = ctypes.c_int
         L.oracle_factgrass.argtypes = [vp, vp, ctypes.c_int, i32, i32, i32, i32, vp, i32, vp, i32,
                                        u32, u32, u64, vp, vp]
+        L.oracle_factgrass_varlen.restype = ctypes.c_int
+        L.oracle_factgrass_varlen.argtypes = [vp, vp, ctypes.c_int, i32, i32, i32, vp, i32, vp, i32, u32, u32, u64,
+                                              vp, vp, vp, vp]
         L.oracle_score.restype = ctypes.c_int
         L.oracle_score.argtypes = [vp, i64, i64, vp, i64, i64, i64, vp, vp]
         L.oracle_num_threads.restype = ctypes.c_int
@@ -136,6 +139,32 @@ def factgrass(A: np.ndarray, G: np.ndarray, mask_in, mask_out, k: int, s: int, s
                                 seed & 0xFFFFFFFFFFFFFFFF, _ptr(out), _ptr(ab))
     if rc:
         raise ValueError(f"oracle_factgrass failed ({rc})")
+    return out, ab
+
+
+def factgrass_varlen(A: np.ndarray, G: np.ndarray, mask_in, mask_out, k: int, s: int, seed: int,
+                     tok_begin, tok_count, dtype: str = "bf16", want_absum: bool = True):
+    """FactGraSS with per-sample sequence lengths.  A: (rows, d_in), G: (rows, d_out); sample b
+    owns rows tok_begin[b] .. tok_begin[b] + tok_count[b] - 1."""
+    _check_data(A, dtype)
+    _check_data(G, dtype)
+    assert A.ndim == 2 and G.ndim == 2 and A.shape[0] == G.shape[0]
+    tok_begin = np.ascontiguousarray(tok_begin, dtype=np.int64)
+    tok_count = np.ascontiguousarray(tok_count, dtype=np.int32)
+    B = tok_begin.size
+    assert tok_count.size == B
+    if B:
+        assert tok_begin.min() >= 0 and tok_count.min() >= 0 and int((tok_begin + tok_count).max()) <= A.shape[0]
+    mask_in = np.ascontiguousarray(mask_in, dtype=np.uint32)
+    mask_out = np.ascontiguousarray(mask_out, dtype=np.uint32)
+    out = np.empty((B, k), dtype=np.float64)
+    ab = np.empty((B, k), dtype=np.float64) if want_absum else None
+    rc = lib().oracle_factgrass_varlen(_ptr(A), _ptr(G), _DT[dtype], B, A.shape[1], G.shape[1], _ptr(mask_in),
+                                       mask_in.size, _ptr(mask_out), mask_out.size, k, s,
+                                       seed & 0xFFFFFFFFFFFFFFFF, _ptr(tok_begin), _ptr(tok_count), _ptr(out),
+                                       _ptr(ab))
+    if rc:
+        raise ValueError(f"oracle_factgrass_varlen failed ({rc})")
     return out, ab
 
 

@@ -242,6 +242,54 @@ int oracle_factgrass(const void *A, const void *G, int dtype, int32_t B, int32_t
     return rc;
 }
 
+/* ---- FactGraSS with per-sample sequence lengths ----------------------------
+ * Eq. 2 sums over the T tokens of ONE sample; samples of a batch have their own
+ * T (the sequence lengths of the paper's Table 3 are maxima).  A and G are
+ * (rows x d_in), (rows x d_out) token-major matrices; the tokens of sample b are
+ * the tok_count[b] consecutive rows starting at row tok_begin[b] (a padded
+ * B x T batch is tok_begin[b] = b*T; a packed batch has no gaps).  Stages 1-3
+ * are those of oracle_factgrass, written out again with the token loop bounded
+ * by the sample's own length.  Pinned by the CPU tests against oracle_factgrass
+ * (full-length, zero-gradient padding, per-sample slices) and against the
+ * materialised projection matrix applied to numpy's A_m^T G_m. */
+int oracle_factgrass_varlen(const void *A, const void *G, int dtype, int32_t B, int32_t d_in,
+                            int32_t d_out, const uint32_t *mask_in, int32_t kin,
+                            const uint32_t *mask_out, int32_t kout, uint32_t k, uint32_t s,
+                            uint64_t seed, const int64_t *tok_begin, const int32_t *tok_count,
+                            double *out, double *absum)
+{
+    if (k == 0 || s == 0 || kin > d_in || kout > d_out || !tok_begin || !tok_count) return 1;
+    const int64_t kp = (int64_t)kin * kout;
+    int rc = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t b = 0; b < B; ++b) {
+        double *gp = (double *)calloc((size_t)(kp > 0 ? kp : 1), sizeof(double));
+        double *ga = (double *)calloc((size_t)(kp > 0 ? kp : 1), sizeof(double));
+        if (!gp || !ga) { rc = 2; free(gp); free(ga); continue; }
+        for (int32_t t = 0; t < tok_count[b]; ++t) {
+            const int64_t row = tok_begin[b] + t;
+            for (int32_t a = 0; a < kin; ++a) {
+                const double x = load_elem(A, dtype, row * d_in + mask_in[a]);      /* a'_t[a] */
+                for (int32_t c = 0; c < kout; ++c) {
+                    const double y = load_elem(G, dtype, row * d_out + mask_out[c]); /* b'_t[c] */
+                    gp[(int64_t)a * kout + c] += x * y;
+                    ga[(int64_t)a * kout + c] += fabs(x * y);
+                }
+            }
+        }
+        double *acc = out + (int64_t)b * k;
+        double *ab = absum ? absum + (int64_t)b * k : NULL;
+        for (uint32_t q = 0; q < k; ++q) { acc[q] = 0.0; if (ab) ab[q] = 0.0; }
+        sjlt_scan(gp, kp, k, s, seed, acc, NULL);
+        if (ab) {
+            double *dump = (double *)calloc(k, sizeof(double));
+            if (dump) { sjlt_scan(ga, kp, k, s, seed, dump, ab); free(dump); } else rc = 2;
+        }
+        free(gp); free(ga);
+    }
+    return rc;
+}
+
 /* ---- attribute-stage score: all-pair inner products (Section 2.1) ---------
  * scores[i*M + m] = <train[i,:], test[m,:]>, absum likewise on |x||y|. */
 int oracle_score(const float *train, int64_t N, int64_t ld_train, const float *test,
