@@ -54,6 +54,7 @@ typedef enum { GRASS_F32 = 0, GRASS_BF16 = 1 } grass_dtype;
 /* bits OR-ed into *dev_status by kernels */
 #define GRASS_DEV_BAD_INDEX 1u   /* a mask index was >= the row length; that element was skipped */
 #define GRASS_DEV_TIMEOUT   2u   /* a bounded on-device wait expired */
+#define GRASS_DEV_BAD_LENGTH 4u  /* a per-sample token count was outside [0, T_max]; it was clamped */
 
 /* SJLT_k with s non-zeros per column of the projection matrix (Section 3.1).  k >= 1, s >= 1. */
 typedef struct {
@@ -116,6 +117,32 @@ grass_status factgrass_compress_grouped(const factgrass_layer* layers /*host*/, 
                                         void* workspace, size_t workspace_bytes,
                                         uint32_t* dev_status, void* stream);
 size_t factgrass_grouped_workspace_bytes(int32_t L);
+
+/*
+ * FactGraSS on batches whose samples have their own sequence lengths.  The sum over tokens in Eq. 2
+ * (Section 3.3.2) runs over the tokens of one sample; padding tokens are not part of it, so they are
+ * not read at all.  A and G of every layer are token-major matrices (rows x d_in, rows x d_out); the
+ * tokens of sample b are the tok_count[b] consecutive rows starting at row tok_begin[b].
+ *   tok_begin  device array of B row indices, or NULL for a padded batch (tok_begin[b] = b * T_max).
+ *   tok_count  device array of B token counts in [0, T_max], or NULL (every sample has T_max tokens).
+ *              A count outside [0, T_max] is clamped and GRASS_DEV_BAD_LENGTH is OR-ed into *dev_status.
+ *   T_max      upper bound of the counts (sizes the launch); with both arrays NULL the calls equal
+ *              factgrass_compress / factgrass_compress_grouped.
+ * A packed batch (no padding rows at all) is tok_begin = exclusive prefix sum of tok_count.
+ * Everything else as in factgrass_compress / factgrass_compress_grouped; a sample with no tokens gets
+ * a zero row.
+ */
+grass_status factgrass_compress_varlen(const void* A, const void* G, grass_dtype dt, int32_t B, int32_t T_max,
+                                       const int64_t* tok_begin, const int32_t* tok_count, int32_t d_in,
+                                       int32_t d_out, const uint32_t* mask_in, int32_t kin,
+                                       const uint32_t* mask_out, int32_t kout,
+                                       const grass_sjlt_spec* spec /*host*/, float* out, int64_t ld_out,
+                                       uint32_t* dev_status, void* stream);
+grass_status factgrass_compress_grouped_varlen(const factgrass_layer* layers /*host*/, int32_t L, grass_dtype dt,
+                                               int32_t B, int32_t T_max, const int64_t* tok_begin,
+                                               const int32_t* tok_count, float* out, int64_t ld_out,
+                                               void* workspace, size_t workspace_bytes,
+                                               uint32_t* dev_status, void* stream);
 
 /*
  * factgrass_compress_grouped for callers that cannot hand over a device workspace.

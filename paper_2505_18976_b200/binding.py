@@ -21,9 +21,10 @@ GRASS_OK = 0
 STATUS = {0: "GRASS_OK", 1: "GRASS_ERR_INVALID_ARG", 2: "GRASS_ERR_BAD_MASK", 3: "GRASS_ERR_UNSUPPORTED",
           4: "GRASS_ERR_CUDA", 5: "GRASS_ERR_TIMEOUT"}
 F32, BF16 = 0, 1
-DEV_BAD_INDEX, DEV_TIMEOUT = 1, 2
+DEV_BAD_INDEX, DEV_TIMEOUT, DEV_BAD_LENGTH = 1, 2, 4
 
 EXPORTS = ("grass_compress", "factgrass_compress", "factgrass_compress_grouped",
+           "factgrass_compress_varlen", "factgrass_compress_grouped_varlen",
            "factgrass_grouped_workspace_bytes", "factgrass_compress_grouped_static", "grass_score", "grass_sjlt_table", "grass_validate_mask",
            "grass_random_mask_host", "grass_status_string")
 
@@ -65,6 +66,12 @@ def lib() -> ctypes.CDLL:
         L.factgrass_compress_grouped.restype = st
         L.factgrass_compress_grouped.argtypes = [ctypes.POINTER(FactgrassLayer), i32, ctypes.c_int, i32, i32, vp, i64,
                                                  vp, ctypes.c_size_t, vp, vp]
+        L.factgrass_compress_varlen.restype = st
+        L.factgrass_compress_varlen.argtypes = [vp, vp, ctypes.c_int, i32, i32, vp, vp, i32, i32, vp, i32, vp, i32, sp,
+                                                vp, i64, vp, vp]
+        L.factgrass_compress_grouped_varlen.restype = st
+        L.factgrass_compress_grouped_varlen.argtypes = [ctypes.POINTER(FactgrassLayer), i32, ctypes.c_int, i32, i32,
+                                                        vp, vp, vp, i64, vp, ctypes.c_size_t, vp, vp]
         L.factgrass_grouped_workspace_bytes.restype = ctypes.c_size_t
         L.factgrass_grouped_workspace_bytes.argtypes = [i32]
         L.factgrass_compress_grouped_static.restype = st
@@ -154,6 +161,39 @@ def factgrass_compress(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, 
     return out
 
 
+def _check_token_arrays(tok_begin, tok_count, B):
+    _need_cuda(tok_begin, tok_count)
+    if tok_begin is not None:
+        assert tok_begin.dtype == torch.int64 and tok_begin.numel() == B and tok_begin.is_contiguous()
+    if tok_count is not None:
+        assert tok_count.dtype == torch.int32 and tok_count.numel() == B and tok_count.is_contiguous()
+
+
+def factgrass_compress_varlen(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, mask_out: torch.Tensor,
+                              k: int, s: int, seed: int, B: int, T_max: int,
+                              tok_begin: Optional[torch.Tensor] = None, tok_count: Optional[torch.Tensor] = None,
+                              out: Optional[torch.Tensor] = None,
+                              dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """One linear layer, samples with their own sequence lengths.  A, G: token-major (rows, d) matrices
+    (or (B, T_max, d) for a padded batch); sample b owns rows tok_begin[b] .. + tok_count[b] (int64 /
+    int32 CUDA tensors; None = b * T_max / T_max)."""
+    _need_cuda(A, G, mask_in, mask_out, out, dev_status)
+    assert A.is_contiguous() and G.is_contiguous()
+    _check_token_arrays(tok_begin, tok_count, B)
+    d_in, d_out = A.shape[-1], G.shape[-1]
+    if tok_begin is None:
+        assert A.numel() >= B * T_max * d_in and G.numel() >= B * T_max * d_out
+    if out is None:
+        out = torch.empty((B, k), dtype=torch.float32, device=A.device)
+    spec = SjltSpec(k, s, seed & 0xFFFFFFFFFFFFFFFF)
+    _check(lib().factgrass_compress_varlen(_ptr(A), _ptr(G), _dt(A), B, T_max, _ptr(tok_begin), _ptr(tok_count),
+                                           d_in, d_out, _ptr(mask_in), mask_in.numel(), _ptr(mask_out),
+                                           mask_out.numel(), ctypes.byref(spec), _ptr(out),
+                                           out.stride(0) if B > 1 else max(out.shape[1], k), _ptr(dev_status),
+                                           _stream()), "factgrass_compress_varlen")
+    return out
+
+
 class GroupedLayers:
     """Host-side descriptor table for factgrass_compress_grouped; keeps the tensors alive."""
 
@@ -188,6 +228,23 @@ def factgrass_compress_grouped(group: GroupedLayers, out: torch.Tensor, workspac
                                             out.stride(0) if out.shape[0] > 1 else out.shape[1], _ptr(workspace),
                                             workspace.numel() * workspace.element_size(), _ptr(dev_status),
                                             _stream()), "factgrass_compress_grouped")
+    return out
+
+
+def factgrass_compress_grouped_varlen(group: GroupedLayers, out: torch.Tensor, workspace: torch.Tensor, B: int,
+                                      T_max: int, tok_begin: Optional[torch.Tensor] = None,
+                                      tok_count: Optional[torch.Tensor] = None,
+                                      dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """All layers of ``group`` in one launch for a batch whose samples have their own lengths; the layers'
+    A and G are token-major (rows, d) matrices that share one token layout (tok_begin, tok_count)."""
+    _need_cuda(out, workspace, dev_status)
+    _check_token_arrays(tok_begin, tok_count, B)
+    assert out.dtype == torch.float32 and out.stride(1) == 1 and out.shape[0] == B
+    _check(lib().factgrass_compress_grouped_varlen(group.array, group.L, group.dtype, B, T_max, _ptr(tok_begin),
+                                                   _ptr(tok_count), _ptr(out),
+                                                   out.stride(0) if out.shape[0] > 1 else out.shape[1],
+                                                   _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                                   _ptr(dev_status), _stream()), "factgrass_compress_grouped_varlen")
     return out
 
 

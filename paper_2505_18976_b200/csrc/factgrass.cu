@@ -58,7 +58,8 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
 template <int TM, int TN>
 __global__ void __launch_bounds__(kFgThreads)
 factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ LayerDesc single, int32_t B,
-                 int32_t T, int32_t max_tiles, int32_t chunk_len, float* __restrict__ out, int64_t ld_out,
+                 int32_t T, const int64_t* __restrict__ tok_begin, const int32_t* __restrict__ tok_count,
+                 int32_t max_tiles, int32_t chunk_len, float* __restrict__ out, int64_t ld_out,
                  uint32_t* dev_status)
 {
     constexpr int PA = TM * 2 + 16;  // smem row pitch in bytes (tokens x masked columns, bf16)
@@ -88,8 +89,19 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     const uint32_t k = L.k;
     const uint32_t s = L.s;
     const uint64_t seed = L.seed;
+    // this sample's tokens: rows [row0, row0 + Tb) of A and G (Tb = T and row0 = b*T without the
+    // per-sample arrays); a length outside [0, T] is clamped and flagged
+    int Tb = T;
+    if (tok_count) {
+        Tb = __ldg(tok_count + b);
+        if (Tb < 0 || Tb > T) {
+            if (dev_status && threadIdx.x == 0 && blockIdx.x == 0) atomicOr(dev_status, GRASS_DEV_BAD_LENGTH);
+            Tb = Tb < 0 ? 0 : T;
+        }
+    }
+    const int64_t row0 = tok_begin ? __ldg(tok_begin + b) : (int64_t)b * T;
     const int t_begin = chunk * chunk_len;
-    const int t_end = min(T, t_begin + chunk_len);
+    const int t_end = min(Tb, t_begin + chunk_len);
     if (t_begin >= t_end) return;
     const bool smem_bins = L.use_smem_bins != 0;
 
@@ -105,8 +117,8 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     uint32_t colG = okG ? __ldg(L.mask_out + tn * TN + gL) : 0u;
     if (okA && colA >= (uint32_t)L.d_in) { bad = true; okA = false; colA = 0; }
     if (okG && colG >= (uint32_t)L.d_out) { bad = true; okG = false; colG = 0; }
-    const uint16_t* pA = L.A + ((int64_t)b * T) * d_in + colA;
-    const uint16_t* pG = L.G + ((int64_t)b * T) * d_out + colG;
+    const uint16_t* pA = L.A + row0 * d_in + colA;
+    const uint16_t* pG = L.G + row0 * d_out + colG;
 
     uint16_t ra[RA], rg[RG];
     auto prefetch = [&](int t0) {
@@ -254,8 +266,8 @@ static int fg_env_int(const char* name, int dflt)
 }
 
 static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, grass_dtype dt, int32_t B, int32_t T,
-                                  float* out, int64_t ld_out, void* workspace, size_t workspace_bytes,
-                                  uint32_t* dev_status, cudaStream_t st)
+                                  const int64_t* tok_begin, const int32_t* tok_count, float* out, int64_t ld_out,
+                                  void* workspace, size_t workspace_bytes, uint32_t* dev_status, cudaStream_t st)
 {
     if (L < 0 || B < 0 || T < 0 || (L > 0 && !layers)) return GRASS_ERR_INVALID_ARG;
     if (dt == GRASS_F32) return GRASS_ERR_UNSUPPORTED;
@@ -347,7 +359,8 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
                 return GRASS_ERR_CUDA;
         }
-        kern<<<grid, kFgThreads, smem, st>>>(dev_descs, single, B, T, max_tiles, chunk_len, out, ld_out, dev_status);
+        kern<<<grid, kFgThreads, smem, st>>>(dev_descs, single, B, T, tok_begin, tok_count, max_tiles, chunk_len, out,
+                                             ld_out, dev_status);
         return launch_status();
     };
     if (tile == 64) return launch(factgrass_kernel<64, 64>, (size_t)kTokTile * (2 * (64 * 2 + 16)));
@@ -373,7 +386,30 @@ extern "C" grass_status factgrass_compress(const void* A, const void* G, grass_d
     l.kout = kout;
     l.spec = *spec;
     l.out_offset = 0;
-    return grass::run_factgrass(&l, 1, dt, B, T, out, ld_out, nullptr, 0, dev_status, (cudaStream_t)stream);
+    return grass::run_factgrass(&l, 1, dt, B, T, nullptr, nullptr, out, ld_out, nullptr, 0, dev_status,
+                                (cudaStream_t)stream);
+}
+
+extern "C" grass_status factgrass_compress_varlen(const void* A, const void* G, grass_dtype dt, int32_t B,
+                                                  int32_t T_max, const int64_t* tok_begin, const int32_t* tok_count,
+                                                  int32_t d_in, int32_t d_out, const uint32_t* mask_in, int32_t kin,
+                                                  const uint32_t* mask_out, int32_t kout, const grass_sjlt_spec* spec,
+                                                  float* out, int64_t ld_out, uint32_t* dev_status, void* stream)
+{
+    if (!spec) return GRASS_ERR_INVALID_ARG;
+    factgrass_layer l;
+    l.A = A;
+    l.G = G;
+    l.mask_in = mask_in;
+    l.mask_out = mask_out;
+    l.d_in = d_in;
+    l.d_out = d_out;
+    l.kin = kin;
+    l.kout = kout;
+    l.spec = *spec;
+    l.out_offset = 0;
+    return grass::run_factgrass(&l, 1, dt, B, T_max, tok_begin, tok_count, out, ld_out, nullptr, 0, dev_status,
+                                (cudaStream_t)stream);
 }
 
 extern "C" size_t factgrass_grouped_workspace_bytes(int32_t L)
@@ -387,8 +423,19 @@ extern "C" grass_status factgrass_compress_grouped(const factgrass_layer* layers
                                                    size_t workspace_bytes, uint32_t* dev_status, void* stream)
 {
     if (!workspace) return GRASS_ERR_INVALID_ARG;
-    return grass::run_factgrass(layers, L, dt, B, T, out, ld_out, workspace, workspace_bytes, dev_status,
-                                (cudaStream_t)stream);
+    return grass::run_factgrass(layers, L, dt, B, T, nullptr, nullptr, out, ld_out, workspace, workspace_bytes,
+                                dev_status, (cudaStream_t)stream);
+}
+
+extern "C" grass_status factgrass_compress_grouped_varlen(const factgrass_layer* layers, int32_t L, grass_dtype dt,
+                                                          int32_t B, int32_t T_max, const int64_t* tok_begin,
+                                                          const int32_t* tok_count, float* out, int64_t ld_out,
+                                                          void* workspace, size_t workspace_bytes,
+                                                          uint32_t* dev_status, void* stream)
+{
+    if (!workspace) return GRASS_ERR_INVALID_ARG;
+    return grass::run_factgrass(layers, L, dt, B, T_max, tok_begin, tok_count, out, ld_out, workspace, workspace_bytes,
+                                dev_status, (cudaStream_t)stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -435,7 +482,7 @@ extern "C" grass_status factgrass_compress_grouped_static(const factgrass_layer*
     void* table = nullptr;
     const grass_status rc = grass::static_table_address(&table);
     if (rc != GRASS_OK) return rc;
-    return grass::run_factgrass(layers, L, dt, B, T, out, ld_out, table,
+    return grass::run_factgrass(layers, L, dt, B, T, nullptr, nullptr, out, ld_out, table,
                                 (size_t)grass::kStaticMaxLayers * sizeof(grass::LayerDesc), dev_status,
                                 (cudaStream_t)stream);
 }
