@@ -185,9 +185,11 @@ class GrassJob:
 class FactJob:
     """configs 3-5: all layers through one factgrass_compress_grouped launch (+ score for config 5)."""
 
-    def __init__(self, cfg, device, G, W):
+    def __init__(self, cfg, device, G, W, seq_len_aware=False):
         self.cfg, self.G, self.device = cfg, G, device
         layers, alg, line = [], 0, 0
+        self.tok_count = None
+        tokens = cfg.B * cfg.T
         self.dense = 0
         self.host_masks = []
         for l, lay in enumerate(cfg.layers):
@@ -196,10 +198,14 @@ class FactJob:
             mi = G.grass_random_mask_host(lay.d_in, cfg.kin, s_in)
             mo = G.grass_random_mask_host(lay.d_out, cfg.kout, s_out)
             self.host_masks.append((mi, mo))
+            if seq_len_aware and self.tok_count is None:
+                # per-sample lengths = tokens before the trailing padding (rows of G that are all zero)
+                self.tok_count = (Gt.abs().amax(dim=2) > 0).int().sum(dim=1).int().contiguous()
+                tokens = int(self.tok_count.sum().item())
             layers.append(dict(A=A, G=Gt, mask_in=G.mask_to_device(mi, device), mask_out=G.mask_to_device(mo, device),
                                k=cfg.k, s=cfg.s, seed=W.layer_hash_seed(cfg, l), out_offset=l * cfg.k))
-            alg += cfg.B * cfg.T * (sector_bytes_per_row(mi, 2) + sector_bytes_per_row(mo, 2)) + cfg.B * cfg.k * 4
-            line += cfg.B * cfg.T * (sector_bytes_per_row(mi, 2, 128) + sector_bytes_per_row(mo, 2, 128)) + cfg.B * cfg.k * 4
+            alg += tokens * (sector_bytes_per_row(mi, 2) + sector_bytes_per_row(mo, 2)) + cfg.B * cfg.k * 4
+            line += tokens * (sector_bytes_per_row(mi, 2, 128) + sector_bytes_per_row(mo, 2, 128)) + cfg.B * cfg.k * 4
             self.dense += cfg.B * cfg.T * (lay.d_in + lay.d_out) * 2
         self.layers = layers
         self.group = G.GroupedLayers(layers)
@@ -224,7 +230,11 @@ class FactJob:
         if ev is not None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-        self.G.factgrass_compress_grouped(self.group, self.out, self.ws)
+        if self.tok_count is not None:
+            self.G.factgrass_compress_grouped_varlen(self.group, self.out, self.ws, self.cfg.B, self.cfg.T,
+                                                     tok_count=self.tok_count)
+        else:
+            self.G.factgrass_compress_grouped(self.group, self.out, self.ws)
         if ev is not None:
             e1.record()
             ev.append((e0, e1))
@@ -237,6 +247,9 @@ class FactJob:
              "k_per_layer": c.k, "l2": self.l2}
         if self.score:
             d["score"] = f"{c.score_n_train}x{c.score_n_test}x{c.k} fp32"
+        if self.tok_count is not None:
+            d["seq_len_aware"] = True
+            d["tokens"] = int(self.tok_count.sum().item())
         return d
 
 
@@ -254,9 +267,9 @@ def small_config(cfg_id, W):
     return cfg
 
 
-def make_job(cfg_id, device, G, W, small=False):
+def make_job(cfg_id, device, G, W, small=False, seq_len_aware=False):
     cfg = small_config(cfg_id, W) if small else W.CONFIGS[cfg_id]
-    return GrassJob(cfg, device, G, W) if cfg_id in (1, 2) else FactJob(cfg, device, G, W)
+    return GrassJob(cfg, device, G, W) if cfg_id in (1, 2) else FactJob(cfg, device, G, W, seq_len_aware)
 
 
 def time_job(job, steps, warmup, world, device):
@@ -454,6 +467,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--small", action="store_true", help="reduced case for profiler captures (not a bench value)")
+    ap.add_argument("--seq-len-aware", action="store_true",
+                    help="configs 3-5: pass per-sample token counts so that padding tokens are not read")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -471,7 +486,7 @@ def main():
     G.lib()
     warmup = args.warmup if args.small else max(args.warmup, 3)
 
-    job = make_job(args.config, device, G, W, small=args.small)
+    job = make_job(args.config, device, G, W, small=args.small, seq_len_aware=args.seq_len_aware)
     sampler = ClockSampler(local)
     sampler.start()
     ms_per_step, dom_ms = time_job(job, args.steps, warmup, world, device)

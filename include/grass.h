@@ -78,11 +78,12 @@ grass_status grass_compress(const void* g, grass_dtype dt, int64_t n, int64_t p,
 /*
  * FactGraSS for one linear layer (Section 3.3.2, stages 1-3; Eq. 2 with selection matrices):
  *   out[b, :] = SJLT( vec( sum_t A[b,t,mask_in] (x) G[b,t,mask_out] ) ),  flat index a*kout + c.
- *   A   B x T x d_in   layer inputs,            token-major contiguous, dtype dt (bf16; see below)
+ *   A   B x T x d_in   layer inputs,            token-major contiguous, dtype dt (bf16 or fp32)
  *   G   B x T x d_out  pre-activation gradients, token-major contiguous, same dtype
  *   out B x spec->k fp32, row stride ld_out.  Overwritten.
- * The kin x kout block is accumulated in fp32 on tensor cores and never reaches memory.
- * dt == GRASS_F32 returns GRASS_ERR_UNSUPPORTED.
+ * The kin x kout block is accumulated in fp32 on tensor cores (tensor memory) and never reaches
+ * HBM.  fp32 factors are split exactly into three bf16 pieces each and contracted with six partial
+ * products, which keeps fp32 accuracy.
  */
 grass_status factgrass_compress(const void* A, const void* G, grass_dtype dt, int32_t B, int32_t T,
                                 int32_t d_in, int32_t d_out, const uint32_t* mask_in, int32_t kin,

@@ -150,7 +150,7 @@ def factgrass_compress(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, 
     assert A.is_contiguous() and G.is_contiguous() and A.dim() == 3 and G.dim() == 3
     B, T, d_in = A.shape
     d_out = G.shape[2]
-    assert G.shape[:2] == (B, T)
+    assert G.shape[:2] == (B, T) and A.dtype == G.dtype
     if out is None:
         out = torch.empty((B, k), dtype=torch.float32, device=A.device)
     spec = SjltSpec(k, s, seed & 0xFFFFFFFFFFFFFFFF)

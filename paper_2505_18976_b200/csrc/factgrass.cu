@@ -12,6 +12,7 @@
 // because SJLT is linear: partial blocks are projected separately and their projections add up in
 // the output row.  Neither the masked factors nor the k'_in x k'_out block ever reach HBM.
 #include "grass_common.cuh"
+#include "tcgen05_util.cuh"
 
 #include <cstdlib>
 #include <cstring>
@@ -23,8 +24,8 @@ constexpr int kFgThreads = 256;
 constexpr int kTokTile = 32;  // tokens per pipeline stage
 
 struct LayerDesc {
-    const uint16_t* A;
-    const uint16_t* G;
+    const void* A;
+    const void* G;
     const uint32_t* mask_in;
     const uint32_t* mask_out;
     int32_t d_in, d_out;
@@ -38,42 +39,45 @@ struct LayerDesc {
 };
 static_assert(sizeof(LayerDesc) == 88, "descriptor layout");
 
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3,
-                                                  uint32_t smem_addr)
+// Token tile staged per pipeline step = the k extent of one shared-memory operand tile.
+static_assert(kTokTile == tc::BK, "a stage holds one operand tile of 32 tokens");
+
+template <bool F32> struct in_elem { using type = uint16_t; };
+template <> struct in_elem<true> { using type = uint32_t; };
+
+// eight consecutive tokens of one masked column (bf16 bit patterns, one per register) -> the 16-byte
+// K-major chunk of that operand row
+__device__ __forceinline__ uint4 pack8_bf16(const uint32_t (&v)[8])
 {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(smem_addr));
+    return make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
 }
 
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// TM x TN block tile of C per CTA; 8 warps as 2 (rows) x 4 (cols).
-template <int TM, int TN>
+// TM x TN block tile of C per CTA (TM = MMA M: masked input coordinates, TN = MMA N: masked output
+// coordinates, contraction over tokens).  F32: fp32 inputs, split exactly into three bf16 pieces.
+template <int TM, int TN, bool F32>
 __global__ void __launch_bounds__(kFgThreads)
 factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ LayerDesc single, int32_t B,
                  int32_t T, const int64_t* __restrict__ tok_begin, const int32_t* __restrict__ tok_count,
                  int32_t max_tiles, int32_t chunk_len, float* __restrict__ out, int64_t ld_out,
                  uint32_t* dev_status)
 {
-    constexpr int PA = TM * 2 + 16;  // smem row pitch in bytes (tokens x masked columns, bf16)
-    constexpr int PG = TN * 2 + 16;
-    constexpr int STAGE = kTokTile * (PA + PG);
-    constexpr int WM = TM / 2, WN = TN / 4;
-    constexpr int MT = WM / 16, NT = WN / 8;
-    constexpr int RA = kTokTile * TM / kFgThreads;  // gathered A elements per thread per stage
-    constexpr int RG = kTokTile * TN / kFgThreads;
-    constexpr int STEP_A = kFgThreads / TM, STEP_G = kFgThreads / TN;
-    static_assert(NT % 2 == 0 && MT >= 1, "warp tile");
+    using elem_t = typename in_elem<F32>::type;
+    constexpr int NP = F32 ? 3 : 1;                       // bf16 pieces per operand
+    constexpr int A_TILE = TM * (int)tc::ROW_BYTES;       // one piece of the A operand tile (TM rows x 32 tokens)
+    constexpr int G_TILE = TN * (int)tc::ROW_BYTES;
+    constexpr int STAGE = NP * (A_TILE + G_TILE);
+    constexpr int NBUF = 2;
+    constexpr int GA = kFgThreads / TM, GG = kFgThreads / TN;   // 8-token groups covered by one pass
+    constexpr int PASS_A = 4 / GA, PASS_G = 4 / GG;             // passes per 32-token stage
+    constexpr uint32_t ACC_COLS = F32 ? 2 * TN : TN;            // fp32 accumulator columns in tensor memory
+    static_assert((TM == 64 || TM == 128) && (TN == 64 || TN == 128), "tile");
+    static_assert(STAGE % 512 == 0, "operand tiles stay 512-byte aligned");
 
-    extern __shared__ __align__(16) unsigned char smem[];
-    float* bins = reinterpret_cast<float*>(smem + 2 * STAGE);
+    extern __shared__ __align__(1024) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long bars[NBUF + 1];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    float* bins = reinterpret_cast<float*>(smem + NBUF * STAGE);
 
     const LayerDesc& L = descs ? descs[blockIdx.z] : single;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -102,119 +106,200 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     const int64_t row0 = tok_begin ? __ldg(tok_begin + b) : (int64_t)b * T;
     const int t_begin = chunk * chunk_len;
     const int t_end = min(Tb, t_begin + chunk_len);
-    if (t_begin >= t_end) return;
+    if (t_begin >= t_end) return;          // whole CTA leaves together, before any barrier or allocation
     const bool smem_bins = L.use_smem_bins != 0;
 
+    const uint32_t bar0 = tc::smem_u32(&bars[0]), bar_done = tc::smem_u32(&bars[NBUF]);
+    if (tid == 0) {
+        for (int i = 0; i < NBUF; ++i) tc::mbar_init(bar0 + 8 * i, 1);
+        tc::mbar_init(bar_done, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc::smem_u32(&tmem_slot)),
+                     "r"(ACC_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
     if (smem_bins)
         for (uint32_t i = tid; i < k; i += kFgThreads) bins[i] = 0.0f;
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = tmem_slot;
 
-    // this thread's gather columns (fixed for the whole chunk)
+    // this thread's gather columns (fixed for the whole chunk): masked coordinate aL of the A tile and
+    // gL of the G tile; per pass it reads 8 consecutive tokens of them (one 16-byte operand chunk)
     bool bad = false;
     const int aL = tid % TM, gL = tid % TN;
-    const int tokA = tid / TM, tokG = tid / TN;
+    const int grpA = tid / TM, grpG = tid / TN;
     bool okA = tm * TM + aL < kin, okG = tn * TN + gL < kout;
     uint32_t colA = okA ? __ldg(L.mask_in + tm * TM + aL) : 0u;
     uint32_t colG = okG ? __ldg(L.mask_out + tn * TN + gL) : 0u;
     if (okA && colA >= (uint32_t)L.d_in) { bad = true; okA = false; colA = 0; }
     if (okG && colG >= (uint32_t)L.d_out) { bad = true; okG = false; colG = 0; }
-    const uint16_t* pA = L.A + row0 * d_in + colA;
-    const uint16_t* pG = L.G + row0 * d_out + colG;
+    const elem_t* pA = reinterpret_cast<const elem_t*>(L.A) + row0 * d_in + colA;
+    const elem_t* pG = reinterpret_cast<const elem_t*>(L.G) + row0 * d_out + colG;
 
-    uint16_t ra[RA], rg[RG];
+    uint32_t ra[PASS_A][8], rg[PASS_G][8];   // gathered elements: fp32 bits, or bf16 bits in the low half
+    auto load1 = [](const elem_t* p) -> uint32_t {
+        if constexpr (F32) return gather_u32(p); else return (uint32_t)gather_u16(p);
+    };
     auto prefetch = [&](int t0) {
 #pragma unroll
-        for (int i = 0; i < RA; ++i) {
-            const int t = t0 + tokA + i * STEP_A;
-            ra[i] = (okA && t < t_end) ? gather_u16(pA + (int64_t)t * d_in) : (uint16_t)0;
-        }
+        for (int ps = 0; ps < PASS_A; ++ps)
 #pragma unroll
-        for (int i = 0; i < RG; ++i) {
-            const int t = t0 + tokG + i * STEP_G;
-            rg[i] = (okG && t < t_end) ? gather_u16(pG + (int64_t)t * d_out) : (uint16_t)0;
+            for (int i = 0; i < 8; ++i) {
+                const int t = t0 + (ps * GA + grpA) * 8 + i;
+                ra[ps][i] = (okA && t < t_end) ? load1(pA + (int64_t)t * d_in) : 0u;
+            }
+#pragma unroll
+        for (int ps = 0; ps < PASS_G; ++ps)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int t = t0 + (ps * GG + grpG) * 8 + i;
+                rg[ps][i] = (okG && t < t_end) ? load1(pG + (int64_t)t * d_out) : 0u;
+            }
+    };
+    // registers -> operand tiles of stage `buf`: row = masked coordinate, 16-byte chunk = 8-token group
+    auto put = [&](unsigned char* tile0, int piece_bytes, int row, int ch, const uint32_t (&v)[8]) {
+        const uint32_t off = tc::operand_chunk_offset(row, ch);
+        if constexpr (F32) {
+            float x[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = __uint_as_float(v[i]);
+            uint4 hi, mid, lo;
+            tc::split8(x, hi, mid, lo);
+            *reinterpret_cast<uint4*>(tile0 + off) = hi;
+            *reinterpret_cast<uint4*>(tile0 + piece_bytes + off) = mid;
+            *reinterpret_cast<uint4*>(tile0 + 2 * piece_bytes + off) = lo;
+        } else {
+            *reinterpret_cast<uint4*>(tile0 + off) = pack8_bf16(v);
         }
     };
     auto stash = [&](int buf) {
         unsigned char* sa = smem + buf * STAGE;
-        unsigned char* sg = sa + kTokTile * PA;
+        unsigned char* sg = sa + NP * A_TILE;
 #pragma unroll
-        for (int i = 0; i < RA; ++i)
-            *reinterpret_cast<uint16_t*>(sa + (tokA + i * STEP_A) * PA + aL * 2) = ra[i];
+        for (int ps = 0; ps < PASS_A; ++ps) put(sa, A_TILE, aL, ps * GA + grpA, ra[ps]);
 #pragma unroll
-        for (int i = 0; i < RG; ++i)
-            *reinterpret_cast<uint16_t*>(sg + (tokG + i * STEP_G) * PG + gL * 2) = rg[i];
+        for (int ps = 0; ps < PASS_G; ++ps) put(sg, G_TILE, gL, ps * GG + grpG, rg[ps]);
     };
 
-    float acc[MT][NT][4];
-#pragma unroll
-    for (int i = 0; i < MT; ++i)
-#pragma unroll
-        for (int j = 0; j < NT; ++j)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.0f;
-
-    const int wm = warp >> 2, wn = warp & 3;
-    const int lm = lane >> 3, lr = lane & 7;  // ldmatrix: matrix id, row within it
-    const uint32_t smem_base = (uint32_t)__cvta_generic_to_shared(smem);
-
+    const uint32_t smem_base = tc::smem_u32(smem);
+    const uint32_t idesc = tc::make_idesc(TM, TN);
+    bool ok = true;
     prefetch(t_begin);
-    int buf = 0;
-    for (int t0 = t_begin; t0 < t_end; t0 += kTokTile, buf ^= 1) {
+    int it = 0;
+    for (int t0 = t_begin; t0 < t_end; t0 += kTokTile, ++it) {
+        const int buf = it % NBUF;
+        // the MMAs that read this buffer two steps ago must have finished before it is overwritten
+        if (it >= NBUF) ok = tc::mbar_wait(bar0 + 8 * buf, (uint32_t)(it / NBUF - 1) & 1u) && ok;
         stash(buf);
-        __syncthreads();
         if (t0 + kTokTile < t_end) prefetch(t0 + kTokTile);
-        const uint32_t sa = smem_base + buf * STAGE;
-        const uint32_t sg = sa + kTokTile * PA;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a0 = smem_base + buf * STAGE, g0 = a0 + NP * A_TILE;
 #pragma unroll
-        for (int k0 = 0; k0 < kTokTile; k0 += 16) {
-            uint32_t af[MT][4];
+            for (int ks = 0; ks < kTokTile / 16; ++ks) {
+                if constexpr (F32) {
+                    // (piece of A, piece of G): 0 = hi, 1 = mid, 2 = lo.  hi*hi goes to the first accumulator,
+                    // the five correction terms to the second (the tensor core truncates after every
+                    // accumulation, so the large sum sees as few of them as possible)
+                    const int pa[6] = {0, 2, 0, 1, 1, 0}, pg[6] = {0, 0, 2, 1, 0, 1};
 #pragma unroll
-            for (int i = 0; i < MT; ++i) {
-                const int row = k0 + (lm >> 1) * 8 + lr;             // token
-                const int colm = wm * WM + i * 16 + (lm & 1) * 8;    // masked input coordinate
-                ldmatrix_x4_trans(af[i][0], af[i][1], af[i][2], af[i][3], sa + row * PA + colm * 2);
-            }
-#pragma unroll
-            for (int j = 0; j < NT; j += 2) {
-                uint32_t b0, b1, b2, b3;
-                const int row = k0 + (lm & 1) * 8 + lr;
-                const int coln = wn * WN + j * 8 + (lm >> 1) * 8;
-                ldmatrix_x4_trans(b0, b1, b2, b3, sg + row * PG + coln * 2);
-#pragma unroll
-                for (int i = 0; i < MT; ++i) {
-                    mma_bf16_16816(acc[i][j], af[i], b0, b1);
-                    mma_bf16_16816(acc[i][j + 1], af[i], b2, b3);
+                    for (int q = 0; q < 6; ++q) {
+                        const uint64_t ad = tc::make_smem_desc(a0 + pa[q] * A_TILE + ks * 32);
+                        const uint64_t gd = tc::make_smem_desc(g0 + pg[q] * G_TILE + ks * 32);
+                        tc::umma_bf16(q == 0 ? tmem_d : tmem_d + TN, ad, gd, idesc, (it > 0 || ks > 0 || q > 1) ? 1u : 0u);
+                    }
+                } else {
+                    tc::umma_bf16(tmem_d, tc::make_smem_desc(a0 + ks * 32), tc::make_smem_desc(g0 + ks * 32), idesc,
+                                  (it > 0 || ks > 0) ? 1u : 0u);
                 }
             }
+            tc::umma_commit(bar0 + 8 * buf);                       // buffer free once these MMAs have read it
+            if (t0 + kTokTile >= t_end) tc::umma_commit(bar_done); // accumulator complete
         }
     }
     if (bad && dev_status) atomicOr(dev_status, GRASS_DEV_BAD_INDEX);
-    __syncthreads();  // bins zeroed by all threads before anyone adds (also closes the last stage)
+    ok = tc::mbar_wait(bar_done, 0) && ok;
+    if (!ok) abort_flag = 1;
+    __syncthreads();
+    ok = abort_flag == 0;
+    if (!ok && tid == 0 && dev_status) atomicOr(dev_status, GRASS_DEV_TIMEOUT);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 
-    // stage 3: SJLT of the block; flat position q = a*kout + c (input-major flattening)
+    // stage 3: SJLT of the block; flat position q = a*kout + c (input-major flattening).
+    // Accumulator row a sits in tensor-memory lane a (TM = 128) or lane (a % 16) + 32 * (a / 16) (TM = 64);
+    // warp w may read lanes 32 * (w % 4) .. + 31; the two warps that share a lane quarter split the columns.
     float* orow = out + (int64_t)b * ld_out + L.out_offset;
     const float scale = 1.0f / sqrtf((float)s);
-#pragma unroll
-    for (int i = 0; i < MT; ++i)
-#pragma unroll
-        for (int j = 0; j < NT; ++j)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float v = acc[i][j][e];
-                const int a = tm * TM + wm * WM + i * 16 + (lane >> 2) + (e >> 1) * 8;
-                const int c = tn * TN + wn * WN + j * 8 + (lane & 3) * 2 + (e & 1);
-                if (a < kin && c < kout && v != 0.0f) {
-                    const uint64_t q = (uint64_t)a * (uint64_t)kout + (uint64_t)c;
-                    for (uint32_t r = 0; r < s; ++r) {
-                        const uint64_t h = sjlt_hash_counter(seed, q * s + r + 1);
-                        const uint32_t bk = sjlt_bucket(h, k);
-                        const float sv = (s == 1) ? sjlt_signed(h, v) : sjlt_signed(h, v) * scale;
-                        if (smem_bins) atomicAdd(&bins[bk], sv);
-                        else atomicAdd(orow + bk, sv);
-                    }
-                }
+    const int quarter = warp & 3;
+    const uint32_t tq = tmem_d + ((uint32_t)(quarter * 32) << 16);
+    auto project = [&](int a, int c, float val) {
+        if (a < kin && c < kout && val != 0.0f) {
+            const uint64_t q = (uint64_t)a * (uint64_t)kout + (uint64_t)c;
+            for (uint32_t r = 0; r < s; ++r) {
+                const uint64_t h = sjlt_hash_counter(seed, q * s + r + 1);
+                const uint32_t bk = sjlt_bucket(h, k);
+                const float sv = (s == 1) ? sjlt_signed(h, val) : sjlt_signed(h, val) * scale;
+                if (smem_bins) atomicAdd(&bins[bk], sv);
+                else atomicAdd(orow + bk, sv);
             }
-    if (smem_bins) {
-        __syncthreads();
+        }
+    };
+    if (ok) {
+        if constexpr (TM == 64) {
+            // 16 rows x 32 columns per warp, 16 values per thread
+            const int c0 = (warp >> 2) * 32;
+            uint32_t v[16];
+            tc::tmem_ld_16x256b_x4(tq + (uint32_t)c0, v);
+            if constexpr (F32) {
+                uint32_t w[16];
+                tc::tmem_ld_16x256b_x4(tq + (uint32_t)(TN + c0), w);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(w[e]));
+            } else {
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            }
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                const int a = tm * TM + quarter * 16 + (lane >> 2) + 8 * ((e & 3) >> 1);
+                const int c = tn * TN + c0 + 8 * (e >> 2) + 2 * (lane & 3) + (e & 1);
+                project(a, c, __uint_as_float(v[e]));
+            }
+        } else {
+            const int a = tm * TM + quarter * 32 + lane;
+#pragma unroll 1
+            for (int c0 = (warp >> 2) * 32; c0 < TN; c0 += 64) {
+                uint32_t v[32];
+                tc::tmem_ld32(tq + (uint32_t)c0, v);
+                if constexpr (F32) {
+                    uint32_t w[32];
+                    tc::tmem_ld32(tq + (uint32_t)(TN + c0), w);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(w[e]));
+                } else {
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                }
+#pragma unroll
+                for (int e = 0; e < 32; ++e) project(a, tn * TN + c0 + e, __uint_as_float(v[e]));
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(ACC_COLS) : "memory");
+    }
+    if (smem_bins && ok) {
         for (uint32_t i = tid; i < k; i += kFgThreads) {
             const float v = bins[i];
             if (v != 0.0f) atomicAdd(orow + i, v);
@@ -240,8 +325,8 @@ static grass_status fill_desc(LayerDesc& d, const factgrass_layer& l, int tile, 
         return GRASS_ERR_INVALID_ARG;
     if (l.out_offset < 0) return GRASS_ERR_INVALID_ARG;
     if ((l.kin > 0 && l.kout > 0 && T > 0) && (!l.A || !l.G || !l.mask_in || !l.mask_out)) return GRASS_ERR_INVALID_ARG;
-    d.A = (const uint16_t*)l.A;
-    d.G = (const uint16_t*)l.G;
+    d.A = l.A;
+    d.G = l.G;
     d.mask_in = l.mask_in;
     d.mask_out = l.mask_out;
     d.d_in = l.d_in;
@@ -270,8 +355,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
                                   void* workspace, size_t workspace_bytes, uint32_t* dev_status, cudaStream_t st)
 {
     if (L < 0 || B < 0 || T < 0 || (L > 0 && !layers)) return GRASS_ERR_INVALID_ARG;
-    if (dt == GRASS_F32) return GRASS_ERR_UNSUPPORTED;
-    if (dt != GRASS_BF16) return GRASS_ERR_INVALID_ARG;
+    if (dt != GRASS_BF16 && dt != GRASS_F32) return GRASS_ERR_INVALID_ARG;
     if (L == 0 || B == 0) return GRASS_OK;
     if (!out) return GRASS_ERR_INVALID_ARG;
     if (L > 65535 || B > 65535) return GRASS_ERR_UNSUPPORTED;
@@ -333,38 +417,43 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
 
-    // token chunks.  Every chunk pays a fixed projection epilogue (tile*tile hashes and a k-bin flush),
-    // so chunks are as long as the machine allows: when there are fewer work items than resident CTA
-    // slots the token sum is split just enough to fill one wave; otherwise just enough for ~8 waves
-    // so that the last, partial wave costs little.
-    const int64_t base_items = (int64_t)L * B * max_tiles;
-    const int64_t slots = (int64_t)sms * (tile == 64 ? 3 : 1);
-    const int min_chunk = 64;
-    int64_t want = base_items < slots ? slots / base_items : (8 * slots + base_items - 1) / base_items;
-    int64_t max_chunks = (T + min_chunk - 1) / min_chunk;
-    if (want > max_chunks) want = max_chunks;
-    if (want < 1) want = 1;
-    int chunk_len = (int)((T + want - 1) / want);
-    chunk_len = (chunk_len + kTokTile - 1) / kTokTile * kTokTile;
-    chunk_len = fg_env_int("FACTGRASS_CHUNK", chunk_len);
-    if (chunk_len < kTokTile) chunk_len = kTokTile;
-    chunk_len = (chunk_len + kTokTile - 1) / kTokTile * kTokTile;
-    const int nchunks = (T + chunk_len - 1) / chunk_len;
-
     const size_t bins_bytes = (size_t)max_k_smem * sizeof(float);
-    dim3 grid((unsigned)(nchunks * max_tiles), (unsigned)B, (unsigned)L);
+    const bool f32 = dt == GRASS_F32;
     auto launch = [&](auto kern, size_t stage_bytes) -> grass_status {
         const size_t smem = 2 * stage_bytes + bins_bytes;
-        if (smem > 48 * 1024) {
+        if (smem > 32 * 1024) {   // static shared memory counts toward the 48 KB default limit too
             if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
                 return GRASS_ERR_CUDA;
         }
+        int per_sm = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kFgThreads, smem) != cudaSuccess || per_sm < 1)
+            per_sm = 1;
+        // token chunks.  Every chunk pays a fixed projection epilogue (tile*tile hashes and a k-bin flush),
+        // so chunks are as long as the machine allows: when there are fewer work items than resident CTA
+        // slots the token sum is split just enough to fill one wave; otherwise just enough for ~8 waves
+        // so that the last, partial wave costs little.
+        const int64_t base_items = (int64_t)L * B * max_tiles;
+        const int64_t slots = (int64_t)sms * per_sm;
+        const int min_chunk = 64;
+        int64_t want = base_items < slots ? slots / base_items : (8 * slots + base_items - 1) / base_items;
+        int64_t max_chunks = (T + min_chunk - 1) / min_chunk;
+        if (want > max_chunks) want = max_chunks;
+        if (want < 1) want = 1;
+        int chunk_len = (int)((T + want - 1) / want);
+        chunk_len = (chunk_len + kTokTile - 1) / kTokTile * kTokTile;
+        chunk_len = fg_env_int("FACTGRASS_CHUNK", chunk_len);
+        if (chunk_len < kTokTile) chunk_len = kTokTile;
+        chunk_len = (chunk_len + kTokTile - 1) / kTokTile * kTokTile;
+        const int nchunks = (T + chunk_len - 1) / chunk_len;
+        dim3 grid((unsigned)(nchunks * max_tiles), (unsigned)B, (unsigned)L);
         kern<<<grid, kFgThreads, smem, st>>>(dev_descs, single, B, T, tok_begin, tok_count, max_tiles, chunk_len, out,
                                              ld_out, dev_status);
         return launch_status();
     };
-    if (tile == 64) return launch(factgrass_kernel<64, 64>, (size_t)kTokTile * (2 * (64 * 2 + 16)));
-    return launch(factgrass_kernel<128, 128>, (size_t)kTokTile * (2 * (128 * 2 + 16)));
+    const size_t piece = (size_t)tile * tc::ROW_BYTES * 2;   // one bf16 piece of the A tile plus one of the G tile
+    if (tile == 64)
+        return f32 ? launch(factgrass_kernel<64, 64, true>, 3 * piece) : launch(factgrass_kernel<64, 64, false>, piece);
+    return f32 ? launch(factgrass_kernel<128, 128, true>, 3 * piece) : launch(factgrass_kernel<128, 128, false>, piece);
 }
 
 }  // namespace grass

@@ -16,13 +16,13 @@
 // Three 72 KB stages of 32 k-values each.  Every mbarrier wait is bounded: if one expires the CTA marks
 // its tile with NaN, still frees its tensor memory, and returns.
 #include "grass_common.cuh"
+#include "tcgen05_util.cuh"
 
 namespace grass {
 namespace tc {
 
 constexpr int BM = 128;            // train rows per CTA (MMA M)
 constexpr int BN = 256;            // test rows per CTA (MMA N, upper bound)
-constexpr int BK = 32;             // k values per stage
 constexpr int STAGES = 3;
 #ifndef GRASS_SCORE_PRODUCERS
 #define GRASS_SCORE_PRODUCERS 512
@@ -40,105 +40,7 @@ constexpr int B_SPLIT_BYTES = BN * BK * 2;   // one bf16 piece of the test tile:
 constexpr int STAGE_BYTES = 3 * (A_SPLIT_BYTES + B_SPLIT_BYTES);   // 72 KB
 constexpr int CHUNKS = BK / 8;     // 16-byte chunks (8 bf16) per row per stage
 constexpr int TASKS = (BM + BN) * CHUNKS / PRODUCERS;   // (row, chunk) tasks per producer per stage = 6
-constexpr uint32_t ROW_BYTES = BK * 2;        // one row of a bf16 piece: 64 bytes = one 64-byte swizzle row
-constexpr uint32_t SBO = 8 * ROW_BYTES;       // bytes between consecutive 8-row groups (512)
-static_assert(ROW_BYTES == 64, "the shared-memory layout below is the 64-byte-swizzle K-major one");
 constexpr uint32_t TMEM_COLS = 512;   // two fp32 accumulators of BN columns each
-constexpr uint32_t SPIN_LIMIT = 1u << 22;
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// bounded wait on the phase with the given parity; false if the limit ran out
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
-{
-    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred P;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, P;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
-    }
-    return false;
-}
-
-// shared-memory matrix descriptor: K-major, 64-byte swizzle, version 1 (sm_100).  Rows are 64 bytes
-// apart, 8-row groups SBO apart; the 16-byte chunk c of row r sits at chunk position c ^ ((r >> 1) & 3)
-// (address bits [4,6) xor bits [7,9)).  The leading-dimension offset is not used by swizzled K-major
-// layouts (set to 16 bytes).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr)
-{
-    return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(SBO >> 4) << 32) | (1ull << 46) |
-           (4ull << 61);
-}
-
-// instruction descriptor: D fp32, A and B bf16, both K-major, M x N
-__device__ __forceinline__ uint32_t make_idesc(uint32_t m, uint32_t n)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((m >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr)
-        : "memory");
-}
-
-// eight consecutive fp32 -> three 16-byte chunks of bf16 (hi, mid, lo), x = hi + mid + lo exactly
-__device__ __forceinline__ void split8(const float (&x)[8], uint4& hi, uint4& mid, uint4& lo)
-{
-    uint32_t h[8], m[8], l[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const uint32_t xb = __float_as_uint(x[i]);
-        h[i] = xb & 0xFFFF0000u;
-        const float r1 = x[i] - __uint_as_float(h[i]);
-        m[i] = __float_as_uint(r1) & 0xFFFF0000u;
-        const float r2 = r1 - __uint_as_float(m[i]);
-        l[i] = __float_as_uint(r2);
-    }
-    hi = make_uint4(__byte_perm(h[0], h[1], 0x7632), __byte_perm(h[2], h[3], 0x7632), __byte_perm(h[4], h[5], 0x7632),
-                    __byte_perm(h[6], h[7], 0x7632));
-    mid = make_uint4(__byte_perm(m[0], m[1], 0x7632), __byte_perm(m[2], m[3], 0x7632), __byte_perm(m[4], m[5], 0x7632),
-                     __byte_perm(m[6], m[7], 0x7632));
-    lo = make_uint4(__byte_perm(l[0], l[1], 0x7632), __byte_perm(l[2], l[3], 0x7632), __byte_perm(l[4], l[5], 0x7632),
-                    __byte_perm(l[6], l[7], 0x7632));
-}
-
 __global__ void __launch_bounds__(THREADS, 1)
 grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_train, const float* __restrict__ test,
                       int64_t M, int64_t ld_test, int64_t D, float* __restrict__ scores, int64_t ld_s, int vec_ok,
@@ -218,7 +120,7 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
                 split8(srcv[q], hi, mid, lo);
                 unsigned char* base = is_a ? st : st + 3 * A_SPLIT_BYTES;
                 const int piece = is_a ? A_SPLIT_BYTES : B_SPLIT_BYTES;
-                const int off = (r >> 3) * SBO + (r & 7) * ROW_BYTES + ((ch ^ ((r >> 1) & 3)) << 4);
+                const uint32_t off = operand_chunk_offset(r, ch);
                 *reinterpret_cast<uint4*>(base + off) = hi;
                 *reinterpret_cast<uint4*>(base + piece + off) = mid;
                 *reinterpret_cast<uint4*>(base + 2 * piece + off) = lo;

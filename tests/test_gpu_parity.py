@@ -200,9 +200,9 @@ def _fact_cfg(W, **kw):
     return W.FactGrassWorkload(**base)
 
 
-def _fact_case(G, W, oracle_mod, cfg, l=0, grouped=False):
+def _fact_case(G, W, oracle_mod, cfg, l=0, grouped=False, dtype=torch.bfloat16):
     lay = cfg.layers[l]
-    A, Gt = W.layer_io(cfg, l, device="cuda")
+    A, Gt = W.layer_io(cfg, l, device="cuda", dtype=dtype)
     s_in, s_out = W.layer_mask_seeds(cfg, l)
     mi = oracle_mod.random_mask(lay.d_in, cfg.kin, s_in)
     mo = oracle_mod.random_mask(lay.d_out, cfg.kout, s_out)
@@ -211,11 +211,13 @@ def _fact_case(G, W, oracle_mod, cfg, l=0, grouped=False):
     out = G.factgrass_compress(A, Gt, _dev_mask(G, mi), _dev_mask(G, mo), cfg.k, cfg.s, seed, dev_status=st)
     torch.cuda.synchronize()
     assert int(st.item()) == 0
-    ref, absum = oracle_mod.factgrass(W.bits_of(A), W.bits_of(Gt), mi, mo, cfg.k, cfg.s, seed)
+    f32 = dtype == torch.float32
+    ref, absum = oracle_mod.factgrass(W.bits_of(A), W.bits_of(Gt), mi, mo, cfg.k, cfg.s, seed,
+                                      dtype="f32" if f32 else "bf16")
     ob, _ = oracle_mod.sjlt_table(cfg.k, cfg.s, seed, cfg.kin * cfg.kout)
     chain = cfg.T + max_bin_load(ob, cfg.k) + 64
-    return check_close(out.cpu().numpy(), ref, absum, TOL_BF16, chain, eps=EPS_TC,
-                       what=f"factgrass {lay} B={cfg.B} T={cfg.T} k'={cfg.kin}x{cfg.kout} k={cfg.k}")
+    return check_close(out.cpu().numpy(), ref, absum, TOL_F32 if f32 else TOL_BF16, chain, eps=EPS_TC,
+                       what=f"factgrass {lay} B={cfg.B} T={cfg.T} k'={cfg.kin}x{cfg.kout} k={cfg.k} {dtype}")
 
 
 @pytest.mark.parametrize("kw", [
@@ -234,6 +236,30 @@ def test_factgrass_parity(G, W, oracle_mod, kw):
     if "layers" in kw and kw["layers"] is None:
         kw["layers"] = (W.LinearLayer("l", 768, 3072),)
     _fact_case(G, W, oracle_mod, _fact_cfg(W, **kw))
+
+
+@pytest.mark.parametrize("kw", [
+    dict(),
+    dict(kin=64, kout=64, k=1024, T=200, B=4),
+    dict(layers=None, kin=128, kout=128, k=4096, T=130, B=3),
+    dict(layers=None, kin=130, kout=260, k=5000, T=64, B=2),
+    dict(kin=24, kout=40, k=97, s=2),
+    dict(kin=64, kout=64, k=256, T=300, pad_frac=0.2, g_dist="laplace"),
+])
+def test_factgrass_fp32_inputs(G, W, oracle_mod, kw):
+    """fp32 factors: the contraction runs on exact bf16 splits and must hold the fp32 tolerance."""
+    kw = dict(kw)
+    if "layers" in kw and kw["layers"] is None:
+        kw["layers"] = (W.LinearLayer("l", 768, 3072),)
+    rel = _fact_case(G, W, oracle_mod, _fact_cfg(W, **kw), dtype=torch.float32)
+    assert rel < 1e-4
+
+
+def test_factgrass_fp32_tile128(G, W, oracle_mod, monkeypatch):
+    monkeypatch.setenv("FACTGRASS_TILE", "128")
+    cfg = _fact_cfg(W, layers=(W.LinearLayer("l", 768, 3072),), kin=128, kout=128, k=4096, T=130, B=3)
+    _fact_case(G, W, oracle_mod, cfg, dtype=torch.float32)
+    _fact_case(G, W, oracle_mod, cfg)
 
 
 @pytest.mark.parametrize("chunk", [32, 64, 1 << 20])
@@ -277,10 +303,9 @@ def test_factgrass_errors_and_empty(G, W, oracle_mod):
     o = torch.full((3, 97), 5.0, device="cuda")
     G.factgrass_compress(A[:, :0].contiguous(), Gt[:, :0].contiguous(), _dev_mask(G, mi), _dev_mask(G, mo), 97, 1, 0, out=o)
     assert torch.all(o == 0)
-    # fp32 inputs: unsupported
-    with pytest.raises(G.GrassError) as e:
-        G.factgrass_compress(A.float(), Gt.float(), _dev_mask(G, mi), _dev_mask(G, mo), 97, 1, 0)
-    assert e.value.code == 3
+    # A and G must have the same dtype
+    with pytest.raises((G.GrassError, AssertionError, TypeError)):
+        G.factgrass_compress(A.float(), Gt, _dev_mask(G, mi), _dev_mask(G, mo), 97, 1, 0)
     # an out-of-range mask index is skipped and flagged
     bad = mo.copy()
     bad[-1] = 4_000_000_000

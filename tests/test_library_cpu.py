@@ -52,8 +52,8 @@ def test_host_side_argument_checks_need_no_gpu(cuda_lib):
     assert L.grass_compress(one, 0, -1, 10, 10, None, 10, ctypes.byref(spec), one, 16, None, None) == INVALID
     assert L.grass_compress(one, 7, 4, 10, 10, None, 10, ctypes.byref(spec), one, 16, None, None) == UNSUPPORTED
     assert L.grass_compress(one, 0, 0, 10, 10, None, 10, ctypes.byref(spec), one, 16, None, None) == 0        # n == 0
-    # FactGraSS: fp32 inputs are not supported, kin > d_in is invalid
-    assert L.factgrass_compress(one, one, 0, 2, 8, 16, 16, one, 4, one, 4, ctypes.byref(spec), one, 16, None, None) == UNSUPPORTED
+    # FactGraSS: an unknown dtype and kin > d_in are invalid
+    assert L.factgrass_compress(one, one, 7, 2, 8, 16, 16, one, 4, one, 4, ctypes.byref(spec), one, 16, None, None) == INVALID
     assert L.factgrass_compress(one, one, 1, 2, 8, 16, 16, one, 17, one, 4, ctypes.byref(spec), one, 16, None, None) == INVALID
     assert L.factgrass_compress(one, one, 1, 2, 8, 16, 16, one, 4, one, 4, None, one, 16, None, None) == INVALID
     assert L.factgrass_compress(one, one, 1, 0, 8, 16, 16, one, 4, one, 4, ctypes.byref(spec), one, 16, None, None) == 0
