@@ -61,6 +61,10 @@ def lib() -> ctypes.CDLL:
                                               vp, vp, vp, vp]
         L.oracle_score.restype = ctypes.c_int
         L.oracle_score.argtypes = [vp, i64, i64, vp, i64, i64, i64, vp, vp]
+        L.oracle_fim.restype = ctypes.c_int
+        L.oracle_fim.argtypes = [vp, i64, i64, i64, vp, vp]
+        L.oracle_fim_solve.restype = ctypes.c_int
+        L.oracle_fim_solve.argtypes = [vp, i64, ctypes.c_double, vp, i64, vp]
         L.oracle_num_threads.restype = ctypes.c_int
         L.oracle_set_num_threads.argtypes = [ctypes.c_int]
         _lib = L
@@ -181,6 +185,33 @@ def score(train: np.ndarray, test: np.ndarray, want_absum: bool = True):
     if rc:
         raise ValueError(f"oracle_score failed ({rc})")
     return sc, ab
+
+
+def fim(X: np.ndarray, want_absum: bool = True):
+    """Projected Fisher information matrix F = X^T X / n of n compressed gradients (rows of X, float32)."""
+    _check_data(X, "f32")
+    n, k = X.shape
+    F = np.empty((k, k), dtype=np.float64)
+    ab = np.empty((k, k), dtype=np.float64) if want_absum else None
+    rc = lib().oracle_fim(_ptr(X), n, k, k, _ptr(F), _ptr(ab))
+    if rc:
+        raise ValueError(f"oracle_fim failed ({rc})")
+    return F, ab
+
+
+def fim_solve(F: np.ndarray, lam: float, Bm: np.ndarray) -> np.ndarray:
+    """Rows x_m = (F + lam I)^-1 b_m for the rows b_m of Bm (float64)."""
+    F = np.ascontiguousarray(F, dtype=np.float64)
+    Bm = np.ascontiguousarray(Bm, dtype=np.float64)
+    k = F.shape[0]
+    assert F.shape == (k, k) and Bm.shape[1] == k
+    X = np.empty_like(Bm)
+    rc = lib().oracle_fim_solve(_ptr(F), k, float(lam), _ptr(Bm), Bm.shape[0], _ptr(X))
+    if rc == 2:
+        raise np.linalg.LinAlgError("F + lambda I is not positive definite")
+    if rc:
+        raise ValueError(f"oracle_fim_solve failed ({rc})")
+    return X
 
 
 def num_threads() -> int:

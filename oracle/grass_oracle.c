@@ -311,6 +311,68 @@ int oracle_score(const float *train, int64_t N, int64_t ld_train, const float *t
     return 0;
 }
 
+/* ---- projected Fisher information matrix and iFVP (Section 2.1, cache stage) ---
+ * F = (1/n) sum_i g_i g_i^T over the n compressed gradients (rows of X, n x k,
+ * row stride ld); with the layer-wise block-diagonal approximation of Section
+ * 3.3.2 this is applied to one layer's k_l columns at a time.  absum is the same
+ * sum over |g_i(a) g_i(b)|. */
+int oracle_fim(const float *X, int64_t n, int64_t k, int64_t ld, double *F, double *absum)
+{
+    if (n <= 0 || k < 0 || ld < k) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t a = 0; a < k; ++a)
+        for (int64_t b = 0; b < k; ++b) {
+            double acc = 0.0, ab = 0.0;
+            for (int64_t i = 0; i < n; ++i) {
+                const double p = (double)X[i * ld + a] * (double)X[i * ld + b];
+                acc += p;
+                ab += fabs(p);
+            }
+            F[a * k + b] = acc / (double)n;
+            if (absum) absum[a * k + b] = ab / (double)n;
+        }
+    return 0;
+}
+
+/* iFVP with damping: x_m = (F + lambda I)^{-1} b_m for the M rows b_m of Bm (M x k).
+ * The paper states the product with the inverse (Section 2.1) and the damping term
+ * (appendix on experiment details); the system is solved here by the textbook Cholesky
+ * factorisation F + lambda I = L L^T, forward substitution L y = b, back substitution
+ * L^T x = y, all in double.  Returns 2 if the matrix is not positive definite. */
+int oracle_fim_solve(const double *F, int64_t k, double lambda, const double *Bm, int64_t M, double *Xout)
+{
+    double *L = (double *)calloc((size_t)(k > 0 ? k * k : 1), sizeof(double));
+    if (!L) return 3;
+    for (int64_t j = 0; j < k; ++j) {
+        double d = F[j * k + j] + lambda;
+        for (int64_t q = 0; q < j; ++q) d -= L[j * k + q] * L[j * k + q];
+        if (!(d > 0.0)) { free(L); return 2; }
+        L[j * k + j] = sqrt(d);
+        for (int64_t i = j + 1; i < k; ++i) {
+            double v = F[i * k + j];
+            for (int64_t q = 0; q < j; ++q) v -= L[i * k + q] * L[j * k + q];
+            L[i * k + j] = v / L[j * k + j];
+        }
+    }
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        double *x = Xout + m * k;
+        const double *b = Bm + m * k;
+        for (int64_t i = 0; i < k; ++i) {                 /* L y = b */
+            double v = b[i];
+            for (int64_t q = 0; q < i; ++q) v -= L[i * k + q] * x[q];
+            x[i] = v / L[i * k + i];
+        }
+        for (int64_t i = k - 1; i >= 0; --i) {            /* L^T x = y */
+            double v = x[i];
+            for (int64_t q = i + 1; q < k; ++q) v -= L[q * k + i] * x[q];
+            x[i] = v / L[i * k + i];
+        }
+    }
+    free(L);
+    return 0;
+}
+
 #ifdef _OPENMP
 #include <omp.h>
 int oracle_num_threads(void) { return omp_get_max_threads(); }
