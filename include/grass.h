@@ -23,6 +23,7 @@
  *   - Zero-size calls (n == 0, B == 0, T == 0 ...) are valid and leave a zeroed / untouched output.
  *   - Mask index lists are uint32, strictly ascending, < p ("exactly one non-repetitive non-zero
  *     entry per row" of the selection matrix, Section 3.2).  They are shared by all samples of a call.
+ *     A NULL mask is the identity and requires the masked length to equal the row length.
  *
  * The sparse projection (Section 3.1) is defined by a seed, not by stored indices.  For input
  * position j (position in the MASKED vector) and draw r < s:
@@ -55,6 +56,7 @@ typedef enum { GRASS_F32 = 0, GRASS_BF16 = 1 } grass_dtype;
 #define GRASS_DEV_BAD_INDEX 1u   /* a mask index was >= the row length; that element was skipped */
 #define GRASS_DEV_TIMEOUT   2u   /* a bounded on-device wait expired */
 #define GRASS_DEV_BAD_LENGTH 4u  /* a per-sample token count was outside [0, T_max]; it was clamped */
+#define GRASS_DEV_NOT_PD    8u   /* grass_fim_factor met a pivot <= 0: F + lambda I is not positive definite */
 
 /* SJLT_k with s non-zeros per column of the projection matrix (Section 3.1).  k >= 1, s >= 1. */
 typedef struct {
@@ -181,6 +183,33 @@ grass_status factgrass_compress_grouped_static(const factgrass_layer* layers /*h
  */
 grass_status grass_score(const float* train, int64_t N, int64_t ld_train, const float* test, int64_t M,
                          int64_t ld_test, int64_t D, float* scores, int64_t ld_s, void* stream);
+
+/*
+ * Projected Fisher information matrix (Section 2.1, cache stage step 2):
+ *   F[a*ld_f + b] = (1/n) * sum_i X[i*ld + a] * X[i*ld + b],   a, b in [0, k).
+ *   X  n x k compressed gradients, fp32, row stride ld >= k (n >= 1).  For the layer-wise block-diagonal
+ *      approximation of Section 3.3.2 pass one layer's column range: X + layer_offset, k = k_l, same ld.
+ *   F  k x k fp32, row stride ld_f >= k.  Overwritten (full symmetric matrix).
+ * The contraction over the n samples runs on tensor cores with fp32 accuracy (exact bf16 splits).
+ */
+grass_status grass_fim(const float* X, int64_t n, int64_t k, int64_t ld, float* F, int64_t ld_f, void* stream);
+
+/*
+ * Damped inverse-FIM-vector products (Section 2.1, cache stage step 3: g~ = F^-1 g; the damping term
+ * lambda is the hyper-parameter of the paper's appendix on experiment details).
+ *   grass_fim_factor  replaces the lower triangle of F by the Cholesky factor L of F + lambda*I
+ *                     (lambda >= 0; the strict upper triangle is left as it was and is not used again).
+ *                     If a pivot is not positive, GRASS_DEV_NOT_PD is OR-ed into *dev_status (nullable)
+ *                     and the result is meaningless; nothing traps.
+ *   grass_fim_apply   overwrites each of the M rows b_m of Bm (M x k fp32, row stride ld_b >= k) by
+ *                     (F + lambda*I)^-1 b_m, using the factor produced by grass_fim_factor.
+ * Preconditioned scores <g_test, F^-1 g_i> = <F^-1 g_test, g_i>: apply to the (few) test rows, then call
+ * grass_score(train, solved_test).  fp32 throughout: the relative error grows with the condition
+ * number of F + lambda*I.
+ */
+grass_status grass_fim_factor(float* F, int64_t k, int64_t ld_f, float lambda, uint32_t* dev_status, void* stream);
+grass_status grass_fim_apply(const float* L, int64_t k, int64_t ld_f, float* Bm, int64_t M, int64_t ld_b,
+                             void* stream);
 
 /*
  * The (bucket, sign) table of SJLT_{k,s,seed} for input positions [0, kprime), produced by the same

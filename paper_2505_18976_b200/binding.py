@@ -21,10 +21,11 @@ GRASS_OK = 0
 STATUS = {0: "GRASS_OK", 1: "GRASS_ERR_INVALID_ARG", 2: "GRASS_ERR_BAD_MASK", 3: "GRASS_ERR_UNSUPPORTED",
           4: "GRASS_ERR_CUDA", 5: "GRASS_ERR_TIMEOUT"}
 F32, BF16 = 0, 1
-DEV_BAD_INDEX, DEV_TIMEOUT, DEV_BAD_LENGTH = 1, 2, 4
+DEV_BAD_INDEX, DEV_TIMEOUT, DEV_BAD_LENGTH, DEV_NOT_PD = 1, 2, 4, 8
 
 EXPORTS = ("grass_compress", "factgrass_compress", "factgrass_compress_grouped",
            "factgrass_compress_varlen", "factgrass_compress_grouped_varlen",
+           "grass_fim", "grass_fim_factor", "grass_fim_apply",
            "factgrass_grouped_workspace_bytes", "factgrass_compress_grouped_static", "grass_score", "grass_sjlt_table", "grass_validate_mask",
            "grass_random_mask_host", "grass_status_string")
 
@@ -79,6 +80,12 @@ def lib() -> ctypes.CDLL:
                                                         i64, vp, vp]
         L.grass_score.restype = st
         L.grass_score.argtypes = [vp, i64, i64, vp, i64, i64, i64, vp, i64, vp]
+        L.grass_fim.restype = st
+        L.grass_fim.argtypes = [vp, i64, i64, i64, vp, i64, vp]
+        L.grass_fim_factor.restype = st
+        L.grass_fim_factor.argtypes = [vp, i64, i64, ctypes.c_float, vp, vp]
+        L.grass_fim_apply.restype = st
+        L.grass_fim_apply.argtypes = [vp, i64, i64, vp, i64, i64, vp]
         L.grass_sjlt_table.restype = st
         L.grass_sjlt_table.argtypes = [sp, i64, vp, vp, vp]
         L.grass_validate_mask.restype = st
@@ -279,6 +286,41 @@ def grass_score(train: torch.Tensor, test: torch.Tensor, out: Optional[torch.Ten
                              test.stride(0) if M > 1 else D, D, _ptr(out), out.stride(0) if N > 1 else M,
                              _stream()), "grass_score")
     return out
+
+
+def grass_fim(X: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """F = X^T X / n for the n rows of X (fp32; a column slice of a wider matrix is fine)."""
+    _need_cuda(X, out)
+    assert X.dtype == torch.float32 and X.dim() == 2 and X.stride(1) == 1
+    n, k = X.shape
+    if out is None:
+        out = torch.empty((k, k), dtype=torch.float32, device=X.device)
+    assert out.dtype == torch.float32 and out.stride(1) == 1 and out.shape == (k, k)
+    _check(lib().grass_fim(_ptr(X), n, k, X.stride(0) if n > 1 else max(k, X.stride(0)), _ptr(out),
+                           out.stride(0) if k > 1 else max(k, 1), _stream()), "grass_fim")
+    return out
+
+
+def grass_fim_factor(F: torch.Tensor, lam: float, dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """In place: lower triangle of F <- Cholesky factor of F + lam * I."""
+    _need_cuda(F, dev_status)
+    assert F.dtype == torch.float32 and F.dim() == 2 and F.shape[0] == F.shape[1] and F.stride(1) == 1
+    k = F.shape[0]
+    _check(lib().grass_fim_factor(_ptr(F), k, F.stride(0) if k > 1 else 1, float(lam), _ptr(dev_status), _stream()),
+           "grass_fim_factor")
+    return F
+
+
+def grass_fim_apply(L: torch.Tensor, Bm: torch.Tensor) -> torch.Tensor:
+    """In place: every row b of Bm <- (L L^T)^-1 b, L from grass_fim_factor."""
+    _need_cuda(L, Bm)
+    assert L.dtype == torch.float32 and Bm.dtype == torch.float32 and Bm.dim() == 2 and Bm.stride(1) == 1
+    k = L.shape[0]
+    assert Bm.shape[1] == k
+    M = Bm.shape[0]
+    _check(lib().grass_fim_apply(_ptr(L), k, L.stride(0) if k > 1 else 1, _ptr(Bm), M,
+                                 Bm.stride(0) if M > 1 else max(k, 1), _stream()), "grass_fim_apply")
+    return Bm
 
 
 def grass_sjlt_table(k: int, s: int, seed: int, kprime: int, device="cuda"):

@@ -35,7 +35,7 @@ struct LayerDesc {
     int64_t out_offset;
     int32_t tiles_m, tiles_n;
     int32_t use_smem_bins;
-    int32_t pad_;
+    float scale;   // raw-block epilogue: factor applied to every entry
 };
 static_assert(sizeof(LayerDesc) == 88, "descriptor layout");
 
@@ -52,9 +52,15 @@ __device__ __forceinline__ uint4 pack8_bf16(const uint32_t (&v)[8])
     return make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
 }
 
+// What happens to the finished k'_in x k'_out block.
+constexpr int kEpiSjlt = 0;   // FactGraSS stage 3: hash every entry into the k-bin accumulator
+constexpr int kEpiRaw = 1;    // add scale * block into a dense symmetric matrix (projected FIM, see grass_fim.cu):
+                              // only tiles on or above the diagonal are computed, the others are mirrored
+
 // TM x TN block tile of C per CTA (TM = MMA M: masked input coordinates, TN = MMA N: masked output
 // coordinates, contraction over tokens).  F32: fp32 inputs, split exactly into three bf16 pieces.
-template <int TM, int TN, bool F32>
+// A NULL mask means the identity (coordinate = position).
+template <int TM, int TN, bool F32, int EPI>
 __global__ void __launch_bounds__(kFgThreads)
 factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ LayerDesc single, int32_t B,
                  int32_t T, const int64_t* __restrict__ tok_begin, const int32_t* __restrict__ tok_count,
@@ -88,6 +94,7 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     const int tile = blockIdx.x % max_tiles;
     const int tm = tile % L.tiles_m, tn = tile / L.tiles_m;
     if (tn >= L.tiles_n) return;
+    if (EPI == kEpiRaw && tn < tm) return;
     const int kin = L.kin, kout = L.kout;
     const int64_t d_in = L.d_in, d_out = L.d_out;
     const uint32_t k = L.k;
@@ -107,7 +114,7 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     const int t_begin = chunk * chunk_len;
     const int t_end = min(Tb, t_begin + chunk_len);
     if (t_begin >= t_end) return;          // whole CTA leaves together, before any barrier or allocation
-    const bool smem_bins = L.use_smem_bins != 0;
+    const bool smem_bins = EPI == kEpiSjlt && L.use_smem_bins != 0;
 
     const uint32_t bar0 = tc::smem_u32(&bars[0]), bar_done = tc::smem_u32(&bars[NBUF]);
     if (tid == 0) {
@@ -135,8 +142,8 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     const int aL = tid % TM, gL = tid % TN;
     const int grpA = tid / TM, grpG = tid / TN;
     bool okA = tm * TM + aL < kin, okG = tn * TN + gL < kout;
-    uint32_t colA = okA ? __ldg(L.mask_in + tm * TM + aL) : 0u;
-    uint32_t colG = okG ? __ldg(L.mask_out + tn * TN + gL) : 0u;
+    uint32_t colA = okA ? (L.mask_in ? __ldg(L.mask_in + tm * TM + aL) : (uint32_t)(tm * TM + aL)) : 0u;
+    uint32_t colG = okG ? (L.mask_out ? __ldg(L.mask_out + tn * TN + gL) : (uint32_t)(tn * TN + gL)) : 0u;
     if (okA && colA >= (uint32_t)L.d_in) { bad = true; okA = false; colA = 0; }
     if (okG && colG >= (uint32_t)L.d_out) { bad = true; okG = false; colG = 0; }
     const elem_t* pA = reinterpret_cast<const elem_t*>(L.A) + row0 * d_in + colA;
@@ -241,7 +248,14 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     const int quarter = warp & 3;
     const uint32_t tq = tmem_d + ((uint32_t)(quarter * 32) << 16);
     auto project = [&](int a, int c, float val) {
-        if (a < kin && c < kout && val != 0.0f) {
+        if constexpr (EPI == kEpiRaw) {
+            // tiles above the diagonal fill their mirror image too; a diagonal tile uses its upper half
+            if (a < kin && c < kout && (tm != tn || a <= c)) {
+                const float sv = val * L.scale;
+                atomicAdd(out + (int64_t)a * ld_out + c, sv);
+                if (a != c) atomicAdd(out + (int64_t)c * ld_out + a, sv);
+            }
+        } else if (a < kin && c < kout && val != 0.0f) {
             const uint64_t q = (uint64_t)a * (uint64_t)kout + (uint64_t)c;
             for (uint32_t r = 0; r < s; ++r) {
                 const uint64_t h = sjlt_hash_counter(seed, q * s + r + 1);
@@ -324,7 +338,8 @@ static grass_status fill_desc(LayerDesc& d, const factgrass_layer& l, int tile, 
     if (l.d_in <= 0 || l.d_out <= 0 || l.kin < 0 || l.kout < 0 || l.kin > l.d_in || l.kout > l.d_out)
         return GRASS_ERR_INVALID_ARG;
     if (l.out_offset < 0) return GRASS_ERR_INVALID_ARG;
-    if ((l.kin > 0 && l.kout > 0 && T > 0) && (!l.A || !l.G || !l.mask_in || !l.mask_out)) return GRASS_ERR_INVALID_ARG;
+    if ((l.kin > 0 && l.kout > 0 && T > 0) && (!l.A || !l.G)) return GRASS_ERR_INVALID_ARG;
+    if ((!l.mask_in && l.kin != l.d_in) || (!l.mask_out && l.kout != l.d_out)) return GRASS_ERR_INVALID_ARG;
     d.A = l.A;
     d.G = l.G;
     d.mask_in = l.mask_in;
@@ -340,7 +355,7 @@ static grass_status fill_desc(LayerDesc& d, const factgrass_layer& l, int tile, 
     d.tiles_m = (l.kin + tile - 1) / tile;
     d.tiles_n = (l.kout + tile - 1) / tile;
     d.use_smem_bins = (size_t)l.spec.k * sizeof(float) <= kMaxSmemBins;
-    d.pad_ = 0;
+    d.scale = 1.0f;
     return GRASS_OK;
 }
 
@@ -452,8 +467,52 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     };
     const size_t piece = (size_t)tile * tc::ROW_BYTES * 2;   // one bf16 piece of the A tile plus one of the G tile
     if (tile == 64)
-        return f32 ? launch(factgrass_kernel<64, 64, true>, 3 * piece) : launch(factgrass_kernel<64, 64, false>, piece);
-    return f32 ? launch(factgrass_kernel<128, 128, true>, 3 * piece) : launch(factgrass_kernel<128, 128, false>, piece);
+        return f32 ? launch(factgrass_kernel<64, 64, true, kEpiSjlt>, 3 * piece)
+                   : launch(factgrass_kernel<64, 64, false, kEpiSjlt>, piece);
+    return f32 ? launch(factgrass_kernel<128, 128, true, kEpiSjlt>, 3 * piece)
+               : launch(factgrass_kernel<128, 128, false, kEpiSjlt>, piece);
+}
+
+// Projected Fisher information matrix F = scale * X^T X of the n rows of X (n x k fp32, row stride ld):
+// the Kronecker-sum contraction of the FactGraSS kernel with both factors = X, identity masks and the
+// raw-block epilogue.  F (k x k, row stride ld_f) must have been zeroed on the stream.
+grass_status launch_fim(const float* X, int64_t n, int64_t k, int64_t ld, float scale, float* F, int64_t ld_f,
+                        cudaStream_t st)
+{
+    constexpr int tile = 128;
+    LayerDesc d;
+    std::memset(&d, 0, sizeof d);
+    d.A = X;
+    d.G = X;
+    d.d_in = d.d_out = (int32_t)ld;
+    d.kin = d.kout = (int32_t)k;
+    d.tiles_m = d.tiles_n = (int32_t)((k + tile - 1) / tile);
+    d.scale = scale;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    auto kern = factgrass_kernel<tile, tile, true, kEpiRaw>;
+    const size_t smem = 2 * 3 * (size_t)tile * tc::ROW_BYTES * 2;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return GRASS_ERR_CUDA;
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kFgThreads, smem) != cudaSuccess || per_sm < 1)
+        per_sm = 1;
+    // sample chunks: enough CTAs for ~4 waves of the tiles on or above the diagonal, at least 256 samples each
+    const int64_t tiles = (int64_t)d.tiles_m * (d.tiles_m + 1) / 2;
+    int64_t want = (4 * (int64_t)sms * per_sm + tiles - 1) / tiles;
+    const int64_t max_chunks = (n + 255) / 256;
+    if (want > max_chunks) want = max_chunks;
+    if (want < 1) want = 1;
+    int64_t chunk_len = (n + want - 1) / want;
+    chunk_len = (chunk_len + kTokTile - 1) / kTokTile * kTokTile;
+    const int64_t nchunks = (n + chunk_len - 1) / chunk_len;
+    const int64_t gx = nchunks * d.tiles_m * d.tiles_n;
+    if (gx > 0x7FFFFFFFLL || chunk_len > 0x7FFFFFFFLL) return GRASS_ERR_UNSUPPORTED;
+    dim3 grid((unsigned)gx, 1, 1);
+    kern<<<grid, kFgThreads, smem, st>>>(nullptr, d, 1, (int32_t)n, nullptr, nullptr, d.tiles_m * d.tiles_n,
+                                         (int32_t)chunk_len, F, ld_f, nullptr);
+    return launch_status();
 }
 
 }  // namespace grass

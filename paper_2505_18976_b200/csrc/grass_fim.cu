@@ -1,0 +1,229 @@
+// Projected Fisher information matrix and damped inverse-FIM-vector products (Section 2.1, cache stage
+// steps 2 and 3; applied per layer block under the block-diagonal approximation of Section 3.3.2).
+//
+//   grass_fim         F = (1/n) sum_i g_i g_i^T over compressed gradients: the tensor-core contraction of
+//                     the FactGraSS kernel with both factors equal to the gradient matrix (factgrass.cu).
+//   grass_fim_factor  F + lambda I = L L^T, blocked right-looking Cholesky in fp32, in place (lower part).
+//   grass_fim_apply   rows b_m <- (L L^T)^-1 b_m by blocked forward and back substitution.
+//
+// The factorisation and the substitutions are plain fp32 FMA kernels on 64-wide blocks: a diagonal-block
+// kernel (one CTA), a row-wise triangular solve against a diagonal block, and a 64 x 64-tile
+// C -= A B^T / C -= A B update.  They are O(k^3) once per layer, next to O(n k^2) for the matrix itself.
+#include "grass_common.cuh"
+
+namespace grass {
+
+grass_status launch_fim(const float* X, int64_t n, int64_t k, int64_t ld, float scale, float* F, int64_t ld_f,
+                        cudaStream_t st);
+
+namespace fim {
+
+constexpr int NB = 64;
+
+__global__ void add_damping_kernel(float* __restrict__ F, int64_t k, int64_t ld, float lambda)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < k) F[i * ld + i] += lambda;
+}
+
+// Unblocked Cholesky of the jb x jb diagonal block at (j0, j0), one CTA.  A pivot that is not positive
+// sets GRASS_DEV_NOT_PD and is replaced by 1 so that nothing divides by zero.
+__global__ void __launch_bounds__(256)
+potrf_diag_kernel(float* __restrict__ F, int64_t ld, int64_t j0, int jb, uint32_t* dev_status)
+{
+    __shared__ float a[NB][NB + 1];
+    const int tid = threadIdx.x;
+    float* blk = F + j0 * ld + j0;
+    for (int e = tid; e < jb * jb; e += 256) {
+        const int i = e / jb, j = e % jb;
+        a[i][j] = (j <= i) ? blk[(int64_t)i * ld + j] : 0.0f;
+    }
+    for (int c = 0; c < jb; ++c) {
+        __syncthreads();
+        float d = a[c][c];
+        if (!(d > 0.0f)) {
+            if (tid == 0 && dev_status) atomicOr(dev_status, GRASS_DEV_NOT_PD);
+            d = 1.0f;
+        }
+        const float sd = sqrtf(d);
+        __syncthreads();
+        if (tid < jb - c) {
+            const int i = c + tid;
+            a[i][c] = (i == c) ? sd : a[i][c] / sd;
+        }
+        __syncthreads();
+        const int m = jb - c - 1;
+        for (int e = tid; e < m * m; e += 256) {
+            const int i = c + 1 + e / m, j = c + 1 + e % m;
+            if (j <= i) a[i][j] -= a[i][c] * a[j][c];
+        }
+    }
+    __syncthreads();
+    for (int e = tid; e < jb * jb; e += 256) {
+        const int i = e / jb, j = e % jb;
+        if (j <= i) blk[(int64_t)i * ld + j] = a[i][j];
+    }
+}
+
+// Rows r of C (rows x jb, at column offset of the block) solved against the diagonal block Ljj (jb x jb,
+// lower):  forward  x Ljj^T = c  (x[q] = (c[q] - sum_{p<q} x[p] L[q][p]) / L[q][q]),
+//          backward x Ljj   = c  (x[q] = (c[q] - sum_{p>q} x[p] L[p][q]) / L[q][q]).
+// One thread per row, 64 rows per CTA.
+template <bool BACKWARD>
+__global__ void __launch_bounds__(NB)
+trsm_rows_kernel(const float* __restrict__ Ljj, int64_t ld_l, int jb, float* __restrict__ C, int64_t ld_c, int64_t rows)
+{
+    __shared__ float l[NB][NB + 1];
+    __shared__ float x[NB][NB + 1];   // x[q][r]
+    const int tid = threadIdx.x;
+    const int64_t r0 = (int64_t)blockIdx.x * NB;
+    for (int e = tid; e < jb * jb; e += NB) {
+        const int i = e / jb, j = e % jb;
+        l[i][j] = (j <= i) ? Ljj[(int64_t)i * ld_l + j] : 0.0f;
+    }
+    for (int rr = 0; rr < NB; ++rr)
+        if (tid < jb) x[tid][rr] = (r0 + rr < rows) ? C[(r0 + rr) * ld_c + tid] : 0.0f;
+    __syncthreads();
+    const int r = tid;
+    if (!BACKWARD) {
+        for (int q = 0; q < jb; ++q) {
+            float v = x[q][r];
+            for (int p = 0; p < q; ++p) v = fmaf(-x[p][r], l[q][p], v);
+            x[q][r] = v / l[q][q];
+        }
+    } else {
+        for (int q = jb - 1; q >= 0; --q) {
+            float v = x[q][r];
+            for (int p = q + 1; p < jb; ++p) v = fmaf(-x[p][r], l[p][q], v);
+            x[q][r] = v / l[q][q];
+        }
+    }
+    __syncthreads();
+    for (int rr = 0; rr < NB; ++rr)
+        if (tid < jb && r0 + rr < rows) C[(r0 + rr) * ld_c + tid] = x[tid][rr];
+}
+
+// C[i][j] -= sum_{q<K} A[i][q] * B(j, q), 64 x 64 tile per CTA, 4 x 4 per thread, K <= 64.
+//   B_TRANS = false: B(j, q) = Bm[j * ldb + q]  (C -= A B^T);  true: B(j, q) = Bm[q * ldb + j]  (C -= A B).
+//   LOWER: C is square, only tiles on or below the diagonal run and only entries j <= i are written.
+template <bool B_TRANS, bool LOWER>
+__global__ void __launch_bounds__(256)
+gemm_sub_kernel(float* __restrict__ C, int64_t ldc, int64_t rows, int64_t cols, const float* __restrict__ A, int64_t lda,
+                const float* __restrict__ Bm, int64_t ldb, int K)
+{
+    if (LOWER && blockIdx.x > blockIdx.y) return;
+    __shared__ __align__(16) float as[NB][NB + 4];   // as[q][i]
+    __shared__ __align__(16) float bs[NB][NB + 4];   // bs[q][j]
+    const int tid = threadIdx.x;
+    const int64_t i0 = (int64_t)blockIdx.y * NB, j0 = (int64_t)blockIdx.x * NB;
+    for (int e = tid; e < NB * NB; e += 256) {
+        const int rr = e / NB, q = e % NB;            // consecutive threads read consecutive q of one row
+        as[q][rr] = (i0 + rr < rows && q < K) ? A[(i0 + rr) * lda + q] : 0.0f;
+        if (!B_TRANS) bs[q][rr] = (j0 + rr < cols && q < K) ? Bm[(j0 + rr) * ldb + q] : 0.0f;
+    }
+    if (B_TRANS)
+        for (int e = tid; e < NB * NB; e += 256) {
+            const int q = e / NB, jj = e % NB;        // consecutive threads read consecutive j of one q
+            bs[q][jj] = (j0 + jj < cols && q < K) ? Bm[(int64_t)q * ldb + j0 + jj] : 0.0f;
+        }
+    __syncthreads();
+    const int ty = tid / 16, tx = tid % 16;
+    float acc[4][4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[u][v] = 0.0f;
+    for (int q = 0; q < K; ++q) {
+        const float4 a4 = *reinterpret_cast<const float4*>(&as[q][ty * 4]);
+        const float4 b4 = *reinterpret_cast<const float4*>(&bs[q][tx * 4]);
+        const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(a[u], b[v], acc[u][v]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int64_t i = i0 + ty * 4 + u;
+        if (i >= rows) continue;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int64_t j = j0 + tx * 4 + v;
+            if (j < cols && (!LOWER || j <= i)) C[i * ldc + j] -= acc[u][v];
+        }
+    }
+}
+
+static inline unsigned blocks(int64_t n) { return (unsigned)((n + NB - 1) / NB); }
+
+}  // namespace fim
+}  // namespace grass
+
+extern "C" grass_status grass_fim(const float* X, int64_t n, int64_t k, int64_t ld, float* F, int64_t ld_f,
+                                  void* stream)
+{
+    if (n <= 0 || k < 0 || ld < k || ld_f < k) return GRASS_ERR_INVALID_ARG;
+    if (k == 0) return GRASS_OK;
+    if (!X || !F) return GRASS_ERR_INVALID_ARG;
+    if (n > 0x7FFFFFFFLL || ld > 0x7FFFFFFFLL) return GRASS_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemset2DAsync(F, (size_t)ld_f * sizeof(float), 0, (size_t)k * sizeof(float), (size_t)k, st) != cudaSuccess)
+        return GRASS_ERR_CUDA;
+    return grass::launch_fim(X, n, k, ld, 1.0f / (float)n, F, ld_f, st);
+}
+
+extern "C" grass_status grass_fim_factor(float* F, int64_t k, int64_t ld_f, float lambda, uint32_t* dev_status,
+                                         void* stream)
+{
+    using namespace grass::fim;
+    if (k < 0 || ld_f < k || !(lambda >= 0.0f)) return GRASS_ERR_INVALID_ARG;
+    if (k == 0) return GRASS_OK;
+    if (!F) return GRASS_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (lambda != 0.0f) add_damping_kernel<<<(unsigned)((k + 255) / 256), 256, 0, st>>>(F, k, ld_f, lambda);
+    for (int64_t j0 = 0; j0 < k; j0 += NB) {
+        const int jb = (int)((k - j0) < NB ? (k - j0) : NB);
+        potrf_diag_kernel<<<1, 256, 0, st>>>(F, ld_f, j0, jb, dev_status);
+        const int64_t rest = k - j0 - jb;
+        if (rest > 0) {
+            float* panel = F + (j0 + jb) * ld_f + j0;            // rows below the diagonal block, its columns
+            trsm_rows_kernel<false><<<blocks(rest), NB, 0, st>>>(F + j0 * ld_f + j0, ld_f, jb, panel, ld_f, rest);
+            float* trail = F + (j0 + jb) * ld_f + (j0 + jb);
+            dim3 g(blocks(rest), blocks(rest));
+            gemm_sub_kernel<false, true><<<g, 256, 0, st>>>(trail, ld_f, rest, rest, panel, ld_f, panel, ld_f, jb);
+        }
+    }
+    return grass::launch_status();
+}
+
+extern "C" grass_status grass_fim_apply(const float* Lf, int64_t k, int64_t ld_f, float* Bm, int64_t M, int64_t ld_b,
+                                        void* stream)
+{
+    using namespace grass::fim;
+    if (k < 0 || M < 0 || ld_f < k || ld_b < k) return GRASS_ERR_INVALID_ARG;
+    if (k == 0 || M == 0) return GRASS_OK;
+    if (!Lf || !Bm) return GRASS_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    // L y = b, block column by block column: solve the diagonal block, then remove its contribution from
+    // the columns to the right
+    for (int64_t j0 = 0; j0 < k; j0 += NB) {
+        const int jb = (int)((k - j0) < NB ? (k - j0) : NB);
+        trsm_rows_kernel<false><<<blocks(M), NB, 0, st>>>(Lf + j0 * ld_f + j0, ld_f, jb, Bm + j0, ld_b, M);
+        const int64_t rest = k - j0 - jb;
+        if (rest > 0) {
+            dim3 g(blocks(rest), blocks(M));
+            gemm_sub_kernel<false, false><<<g, 256, 0, st>>>(Bm + j0 + jb, ld_b, M, rest, Bm + j0, ld_b,
+                                                              Lf + (j0 + jb) * ld_f + j0, ld_f, jb);
+        }
+    }
+    // L^T x = y, from the last block column to the first
+    for (int64_t j0 = ((k - 1) / NB) * NB; j0 >= 0; j0 -= NB) {
+        const int jb = (int)((k - j0) < NB ? (k - j0) : NB);
+        trsm_rows_kernel<true><<<blocks(M), NB, 0, st>>>(Lf + j0 * ld_f + j0, ld_f, jb, Bm + j0, ld_b, M);
+        if (j0 > 0) {
+            dim3 g(blocks(j0), blocks(M));
+            gemm_sub_kernel<true, false><<<g, 256, 0, st>>>(Bm, ld_b, M, j0, Bm + j0, ld_b, Lf + j0 * ld_f, ld_f, jb);
+        }
+    }
+    return grass::launch_status();
+}
