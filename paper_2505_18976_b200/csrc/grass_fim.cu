@@ -68,39 +68,44 @@ potrf_diag_kernel(float* __restrict__ F, int64_t ld, int64_t j0, int jb, uint32_
 // Rows r of C (rows x jb, at column offset of the block) solved against the diagonal block Ljj (jb x jb,
 // lower):  forward  x Ljj^T = c  (x[q] = (c[q] - sum_{p<q} x[p] L[q][p]) / L[q][q]),
 //          backward x Ljj   = c  (x[q] = (c[q] - sum_{p>q} x[p] L[p][q]) / L[q][q]).
-// One thread per row, 64 rows per CTA.
+// One thread per row for the substitution, 64 rows per CTA; all 256 threads move the data.
 template <bool BACKWARD>
-__global__ void __launch_bounds__(NB)
+__global__ void __launch_bounds__(256)
 trsm_rows_kernel(const float* __restrict__ Ljj, int64_t ld_l, int jb, float* __restrict__ C, int64_t ld_c, int64_t rows)
 {
     __shared__ float l[NB][NB + 1];
     __shared__ float x[NB][NB + 1];   // x[q][r]
     const int tid = threadIdx.x;
     const int64_t r0 = (int64_t)blockIdx.x * NB;
-    for (int e = tid; e < jb * jb; e += NB) {
-        const int i = e / jb, j = e % jb;
-        l[i][j] = (j <= i) ? Ljj[(int64_t)i * ld_l + j] : 0.0f;
-    }
-    for (int rr = 0; rr < NB; ++rr)
-        if (tid < jb) x[tid][rr] = (r0 + rr < rows) ? C[(r0 + rr) * ld_c + tid] : 0.0f;
-    __syncthreads();
-    const int r = tid;
-    if (!BACKWARD) {
-        for (int q = 0; q < jb; ++q) {
-            float v = x[q][r];
-            for (int p = 0; p < q; ++p) v = fmaf(-x[p][r], l[q][p], v);
-            x[q][r] = v / l[q][q];
-        }
-    } else {
-        for (int q = jb - 1; q >= 0; --q) {
-            float v = x[q][r];
-            for (int p = q + 1; p < jb; ++p) v = fmaf(-x[p][r], l[p][q], v);
-            x[q][r] = v / l[q][q];
-        }
+#pragma unroll 4
+    for (int e = tid; e < NB * NB; e += 256) {
+        const int i = e / NB, j = e % NB;             // consecutive threads read consecutive columns
+        l[i][j] = (i < jb && j <= i) ? Ljj[(int64_t)i * ld_l + j] : 0.0f;
+        x[j][i] = (j < jb && r0 + i < rows) ? C[(r0 + i) * ld_c + j] : 0.0f;
     }
     __syncthreads();
-    for (int rr = 0; rr < NB; ++rr)
-        if (tid < jb && r0 + rr < rows) C[(r0 + rr) * ld_c + tid] = x[tid][rr];
+    if (tid < NB) {
+        const int r = tid;
+        if (!BACKWARD) {
+            for (int q = 0; q < jb; ++q) {
+                float v = x[q][r];
+                for (int p = 0; p < q; ++p) v = fmaf(-x[p][r], l[q][p], v);
+                x[q][r] = v / l[q][q];
+            }
+        } else {
+            for (int q = jb - 1; q >= 0; --q) {
+                float v = x[q][r];
+                for (int p = q + 1; p < jb; ++p) v = fmaf(-x[p][r], l[p][q], v);
+                x[q][r] = v / l[q][q];
+            }
+        }
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int e = tid; e < NB * NB; e += 256) {
+        const int i = e / NB, j = e % NB;
+        if (j < jb && r0 + i < rows) C[(r0 + i) * ld_c + j] = x[j][i];
+    }
 }
 
 // C[i][j] -= sum_{q<K} A[i][q] * B(j, q), 64 x 64 tile per CTA, 4 x 4 per thread, K <= 64.
@@ -187,7 +192,7 @@ extern "C" grass_status grass_fim_factor(float* F, int64_t k, int64_t ld_f, floa
         const int64_t rest = k - j0 - jb;
         if (rest > 0) {
             float* panel = F + (j0 + jb) * ld_f + j0;            // rows below the diagonal block, its columns
-            trsm_rows_kernel<false><<<blocks(rest), NB, 0, st>>>(F + j0 * ld_f + j0, ld_f, jb, panel, ld_f, rest);
+            trsm_rows_kernel<false><<<blocks(rest), 256, 0, st>>>(F + j0 * ld_f + j0, ld_f, jb, panel, ld_f, rest);
             float* trail = F + (j0 + jb) * ld_f + (j0 + jb);
             dim3 g(blocks(rest), blocks(rest));
             gemm_sub_kernel<false, true><<<g, 256, 0, st>>>(trail, ld_f, rest, rest, panel, ld_f, panel, ld_f, jb);
@@ -208,7 +213,7 @@ extern "C" grass_status grass_fim_apply(const float* Lf, int64_t k, int64_t ld_f
     // the columns to the right
     for (int64_t j0 = 0; j0 < k; j0 += NB) {
         const int jb = (int)((k - j0) < NB ? (k - j0) : NB);
-        trsm_rows_kernel<false><<<blocks(M), NB, 0, st>>>(Lf + j0 * ld_f + j0, ld_f, jb, Bm + j0, ld_b, M);
+        trsm_rows_kernel<false><<<blocks(M), 256, 0, st>>>(Lf + j0 * ld_f + j0, ld_f, jb, Bm + j0, ld_b, M);
         const int64_t rest = k - j0 - jb;
         if (rest > 0) {
             dim3 g(blocks(rest), blocks(M));
@@ -219,7 +224,7 @@ extern "C" grass_status grass_fim_apply(const float* Lf, int64_t k, int64_t ld_f
     // L^T x = y, from the last block column to the first
     for (int64_t j0 = ((k - 1) / NB) * NB; j0 >= 0; j0 -= NB) {
         const int jb = (int)((k - j0) < NB ? (k - j0) : NB);
-        trsm_rows_kernel<true><<<blocks(M), NB, 0, st>>>(Lf + j0 * ld_f + j0, ld_f, jb, Bm + j0, ld_b, M);
+        trsm_rows_kernel<true><<<blocks(M), 256, 0, st>>>(Lf + j0 * ld_f + j0, ld_f, jb, Bm + j0, ld_b, M);
         if (j0 > 0) {
             dim3 g(blocks(j0), blocks(M));
             gemm_sub_kernel<true, false><<<g, 256, 0, st>>>(Bm, ld_b, M, j0, Bm + j0, ld_b, Lf + j0 * ld_f, ld_f, jb);
