@@ -14,6 +14,7 @@
 #include "grass_common.cuh"
 #include "tcgen05_util.cuh"
 
+#include <algorithm>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -436,18 +437,41 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     const bool f32 = dt == GRASS_F32;
     auto launch = [&](auto kern, size_t stage_bytes) -> grass_status {
         const size_t smem = 2 * stage_bytes + bins_bytes;
-        if (smem > 32 * 1024) {   // static shared memory counts toward the 48 KB default limit too
-            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-                return GRASS_ERR_CUDA;
+        // static shared memory counts toward the 48 KB default limit too
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return GRASS_ERR_CUDA;
+        cudaFuncAttributes fa;
+        if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return GRASS_ERR_CUDA;
+        const size_t cta_smem = smem + fa.sharedSizeBytes + 1024;   // + the per-CTA reservation
+        // resident CTAs per SM from the kernel's own footprint: registers, threads, tensor-memory columns
+        // (which the runtime's occupancy query does not count) and shared memory
+        auto resident = [&](size_t smem_per_sm) {
+            int r = 65536 / (fa.numRegs > 0 ? fa.numRegs * kFgThreads : 65536);
+            r = std::min(r, 2048 / kFgThreads);
+            r = std::min(r, 512 / (tile * (f32 ? 2 : 1)));
+            r = std::min(r, (int)(smem_per_sm / cta_smem));
+            return r < 1 ? 1 : r;
+        };
+        const int64_t base_items = (int64_t)L * B * max_tiles;
+        // Gathered loads are tracked in L1 while in flight, so a launch of several waves (the HBM-streaming
+        // regime) runs faster with a small shared-memory carve-out and fewer resident CTAs; a launch of about
+        // one wave wants every CTA slot it can get and keeps the driver's default split.
+        int carve = cudaSharedmemCarveoutDefault, per_sm = resident(227 * 1024);
+        {
+            const size_t small = std::max<size_t>(64 * 1024, cta_smem);
+            const int r_small = resident(small);
+            if (base_items >= 2 * (int64_t)sms * r_small) {
+                per_sm = r_small;
+                carve = cta_smem <= 57 * 1024 ? 25 : (int)((cta_smem * 100 + 228 * 1024 - 1) / (228 * 1024));
+            }
         }
-        int per_sm = 1;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kFgThreads, smem) != cudaSuccess || per_sm < 1)
-            per_sm = 1;
+        carve = fg_env_int("FACTGRASS_CARVEOUT", carve);
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, carve) != cudaSuccess)
+            return GRASS_ERR_CUDA;
         // token chunks.  Every chunk pays a fixed projection epilogue (tile*tile hashes and a k-bin flush),
         // so chunks are as long as the machine allows: when there are fewer work items than resident CTA
         // slots the token sum is split just enough to fill one wave; otherwise just enough for ~8 waves
         // so that the last, partial wave costs little.
-        const int64_t base_items = (int64_t)L * B * max_tiles;
         const int64_t slots = (int64_t)sms * per_sm;
         const int min_chunk = 64;
         int64_t want = base_items < slots ? slots / base_items : (8 * slots + base_items - 1) / base_items;
@@ -495,9 +519,7 @@ grass_status launch_fim(const float* X, int64_t n, int64_t k, int64_t ld, float 
     const size_t smem = 2 * 3 * (size_t)tile * tc::ROW_BYTES * 2;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return GRASS_ERR_CUDA;
-    int per_sm = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kFgThreads, smem) != cudaSuccess || per_sm < 1)
-        per_sm = 1;
+    const int per_sm = 2;   // 97 KB of shared memory and 256 tensor-memory columns per CTA
     // sample chunks: enough CTAs for ~4 waves of the tiles on or above the diagonal, at least 256 samples each
     const int64_t tiles = (int64_t)d.tiles_m * (d.tiles_m + 1) / 2;
     int64_t want = (4 * (int64_t)sms * per_sm + tiles - 1) / tiles;
