@@ -530,8 +530,8 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel per launch, from ncu captures
 # summarised under profiles/ (bytes; None until captured)
-TRAFFIC = {1: 65_797_632 + 326_400, 2: 8 * (425_576_704 + 3_593_984), 3: 124_362_496 + 4_034_048, 4: None,
-           5: 16 * (1_191_473_000 + 5_273_600)}
+TRAFFIC = {1: 65_797_632 + 326_400, 2: 8 * (425_576_704 + 3_593_984), 3: 124_360_704 + 4_261_888,
+           4: 3 * (1_354_085_000 + 4_346_368), 5: 16 * (1_191_550_000 + 5_442_560)}
 
 if __name__ == "__main__":
     main()
