@@ -413,7 +413,7 @@ def oracle_sample(cfg_id, W, budget="baseline"):
     return run, cfg.B * frac, f"first {nl} of {len(cfg.layers)} layers, all {cfg.B} samples x {cfg.T} tokens"
 
 
-def cpu_baseline(cfg_id, W, min_seconds=10.0, max_repeats=50):
+def cpu_baseline(cfg_id, W, min_seconds=10.0, max_repeats=20000):
     """The oracle on the bounded sample, repeated until about `min_seconds` of wall time."""
     import oracle
     oracle.build()
