@@ -185,15 +185,17 @@ class GrassJob:
 class FactJob:
     """configs 3-5: all layers through one factgrass_compress_grouped launch (+ score for config 5)."""
 
-    def __init__(self, cfg, device, G, W, seq_len_aware=False):
+    def __init__(self, cfg, device, G, W, seq_len_aware=False, fp32_inputs=False, precondition=False):
         self.cfg, self.G, self.device = cfg, G, device
+        self.fp32 = fp32_inputs
+        eb = 4 if fp32_inputs else 2
         layers, alg, line = [], 0, 0
         self.tok_count = None
         tokens = cfg.B * cfg.T
         self.dense = 0
         self.host_masks = []
         for l, lay in enumerate(cfg.layers):
-            A, Gt = W.layer_io(cfg, l, device=device)
+            A, Gt = W.layer_io(cfg, l, device=device, dtype=torch.float32 if fp32_inputs else torch.bfloat16)
             s_in, s_out = W.layer_mask_seeds(cfg, l)
             mi = G.grass_random_mask_host(lay.d_in, cfg.kin, s_in)
             mo = G.grass_random_mask_host(lay.d_out, cfg.kout, s_out)
@@ -204,9 +206,9 @@ class FactJob:
                 tokens = int(self.tok_count.sum().item())
             layers.append(dict(A=A, G=Gt, mask_in=G.mask_to_device(mi, device), mask_out=G.mask_to_device(mo, device),
                                k=cfg.k, s=cfg.s, seed=W.layer_hash_seed(cfg, l), out_offset=l * cfg.k))
-            alg += tokens * (sector_bytes_per_row(mi, 2) + sector_bytes_per_row(mo, 2)) + cfg.B * cfg.k * 4
-            line += tokens * (sector_bytes_per_row(mi, 2, 128) + sector_bytes_per_row(mo, 2, 128)) + cfg.B * cfg.k * 4
-            self.dense += cfg.B * cfg.T * (lay.d_in + lay.d_out) * 2
+            alg += tokens * (sector_bytes_per_row(mi, eb) + sector_bytes_per_row(mo, eb)) + cfg.B * cfg.k * 4
+            line += tokens * (sector_bytes_per_row(mi, eb, 128) + sector_bytes_per_row(mo, eb, 128)) + cfg.B * cfg.k * 4
+            self.dense += cfg.B * cfg.T * (lay.d_in + lay.d_out) * eb
         self.layers = layers
         self.group = G.GroupedLayers(layers)
         self.out = torch.empty((cfg.B, cfg.out_dim), dtype=torch.float32, device=device)
@@ -215,12 +217,19 @@ class FactJob:
         if cfg.score_n_train:
             self.score = W.score_vectors(cfg.score_n_train, cfg.score_n_test, cfg.k, cfg.data_seed + 7, device=device)
             self.score_out = torch.empty((cfg.score_n_train, cfg.score_n_test), dtype=torch.float32, device=device)
+        # --precondition: the attribute stage with the damped inverse of the projected FIM of the train vectors
+        # (one layer block): F = train^T train / n, Cholesky of F + lambda I, solve for the test rows, then scores
+        self.precondition = bool(precondition and self.score)
+        if self.precondition:
+            self.fim = torch.empty((cfg.k, cfg.k), dtype=torch.float32, device=device)
+            self.test_pre = torch.empty_like(self.score[1])
         self.samples_per_step = cfg.B
         self.alg_bytes_per_launch = alg
         self.line_bytes_per_launch = line
         self.dense_bytes_per_launch = self.dense
         self.launches_per_step = 1
-        self.kernels_per_step = 2 + (1 if self.score else 0)
+        nb = (cfg.k + 63) // 64
+        self.kernels_per_step = 2 + (1 if self.score else 0) + ((2 + 3 * nb + 4 * nb) if self.precondition else 0)
         self.dominant = "factgrass_kernel"
         self.need_flush = self.dense < 4 * L2_BYTES
         self.l2 = "L2 flushed between steps" if self.need_flush else "inputs >> L2"
@@ -238,7 +247,13 @@ class FactJob:
         if ev is not None:
             e1.record()
             ev.append((e0, e1))
-        if self.score:
+        if self.precondition:
+            self.G.grass_fim(self.score[0], out=self.fim)
+            self.G.grass_fim_factor(self.fim, 0.1)
+            self.test_pre.copy_(self.score[1])
+            self.G.grass_fim_apply(self.fim, self.test_pre)
+            self.G.grass_score(self.score[0], self.test_pre, out=self.score_out)
+        elif self.score:
             self.G.grass_score(self.score[0], self.score[1], out=self.score_out)
 
     def desc(self):
@@ -247,6 +262,10 @@ class FactJob:
              "k_per_layer": c.k, "l2": self.l2}
         if self.score:
             d["score"] = f"{c.score_n_train}x{c.score_n_test}x{c.k} fp32"
+        if self.fp32:
+            d["inputs"] = "fp32"
+        if self.precondition:
+            d["score"] += ", preconditioned by the damped projected FIM (lambda 0.1)"
         if self.tok_count is not None:
             d["seq_len_aware"] = True
             d["tokens"] = int(self.tok_count.sum().item())
@@ -267,9 +286,11 @@ def small_config(cfg_id, W):
     return cfg
 
 
-def make_job(cfg_id, device, G, W, small=False, seq_len_aware=False):
+def make_job(cfg_id, device, G, W, small=False, seq_len_aware=False, fp32_inputs=False, precondition=False):
     cfg = small_config(cfg_id, W) if small else W.CONFIGS[cfg_id]
-    return GrassJob(cfg, device, G, W) if cfg_id in (1, 2) else FactJob(cfg, device, G, W, seq_len_aware)
+    if cfg_id in (1, 2):
+        return GrassJob(cfg, device, G, W)
+    return FactJob(cfg, device, G, W, seq_len_aware, fp32_inputs, precondition)
 
 
 def time_job(job, steps, warmup, world, device):
@@ -467,6 +488,9 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--small", action="store_true", help="reduced case for profiler captures (not a bench value)")
+    ap.add_argument("--fp32-inputs", action="store_true", help="configs 3-5: fp32 A and G instead of bf16")
+    ap.add_argument("--precondition", action="store_true",
+                    help="config 5: projected FIM of the train vectors, damped solve for the test vectors, then scores")
     ap.add_argument("--seq-len-aware", action="store_true",
                     help="configs 3-5: pass per-sample token counts so that padding tokens are not read")
     args = ap.parse_args()
@@ -486,7 +510,10 @@ def main():
     G.lib()
     warmup = args.warmup if args.small else max(args.warmup, 3)
 
-    job = make_job(args.config, device, G, W, small=args.small, seq_len_aware=args.seq_len_aware)
+    job = make_job(args.config, device, G, W, small=args.small, seq_len_aware=args.seq_len_aware,
+                   fp32_inputs=args.fp32_inputs, precondition=args.precondition)
+    if args.fp32_inputs or args.precondition:
+        args.no_e2e = True      # the host-buffer leg covers the default path only
     sampler = ClockSampler(local)
     sampler.start()
     ms_per_step, dom_ms = time_job(job, args.steps, warmup, world, device)
@@ -502,7 +529,7 @@ def main():
                 "line128_bytes_per_launch": int(job.line_bytes_per_launch),
                 "line128_achieved": job.line_bytes_per_launch / (dom_ms * 1e-3) / 1e9,
                 "line128_frac": job.line_bytes_per_launch / (dom_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                "traffic": TRAFFIC.get(args.config)}
+                "traffic": None if (args.fp32_inputs or args.seq_len_aware or args.small) else TRAFFIC.get(args.config)}
 
     e2e = None
     if not args.no_e2e:
@@ -518,7 +545,7 @@ def main():
             cfgd["small"] = True
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
                 "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                "dtype": "bf16" if args.config >= 3 else "f32", "data": "synthetic", "config": cfgd,
+                "dtype": "bf16" if (args.config >= 3 and not args.fp32_inputs) else "f32", "data": "synthetic", "config": cfgd,
                 "tokens_per_s": (value * job.cfg.T if args.config >= 3 else None),
                 "clocks": clocks, "e2e": e2e, "gpu_launches": job.kernels_per_step * args.steps,
                 "roofline": roofline, "cpu_baseline": cpu}

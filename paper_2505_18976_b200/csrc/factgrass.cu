@@ -453,17 +453,19 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
             return r < 1 ? 1 : r;
         };
         const int64_t base_items = (int64_t)L * B * max_tiles;
-        // Gathered loads are tracked in L1 while in flight, so a launch of several waves (the HBM-streaming
-        // regime) runs faster with a small shared-memory carve-out and fewer resident CTAs; a launch of about
-        // one wave wants every CTA slot it can get and keeps the driver's default split.
-        int carve = cudaSharedmemCarveoutDefault, per_sm = resident(227 * 1024);
+        // Gathered loads are tracked in L1 while in flight, and L1 is what the shared-memory carve-out leaves
+        // of the SM's 256 KB.  A launch of several waves (the HBM-streaming regime) runs fastest with one to
+        // three resident CTAs and a 64 KB carve-out; a launch of about one wave wants more CTA slots but still
+        // keeps about 90 KB of L1 (carve-out at most 164 KB).  The driver's default would size the carve-out
+        // for the largest number of CTAs and starve L1.
+        const bool streaming = base_items >= 2 * (int64_t)sms * resident(std::max<size_t>(64 * 1024, cta_smem));
+        const size_t cap = std::max<size_t>((streaming ? 64 : 164) * 1024, cta_smem);
+        int per_sm = resident(cap);
+        int carve = 100;
         {
-            const size_t small = std::max<size_t>(64 * 1024, cta_smem);
-            const int r_small = resident(small);
-            if (base_items >= 2 * (int64_t)sms * r_small) {
-                per_sm = r_small;
-                carve = cta_smem <= 57 * 1024 ? 25 : (int)((cta_smem * 100 + 228 * 1024 - 1) / (228 * 1024));
-            }
+            const int configs_kb[] = {8, 16, 32, 64, 100, 132, 164, 196, 228};
+            for (int kb : configs_kb)
+                if ((size_t)kb * 1024 >= (size_t)per_sm * cta_smem) { carve = kb * 100 / 228; break; }
         }
         carve = fg_env_int("FACTGRASS_CARVEOUT", carve);
         if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, carve) != cudaSuccess)
@@ -519,7 +521,9 @@ grass_status launch_fim(const float* X, int64_t n, int64_t k, int64_t ld, float 
     const size_t smem = 2 * 3 * (size_t)tile * tc::ROW_BYTES * 2;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return GRASS_ERR_CUDA;
-    const int per_sm = 2;   // 97 KB of shared memory and 256 tensor-memory columns per CTA
+    const int per_sm = 2;   // 97 KB of shared memory and 256 tensor-memory columns per CTA; 196 KB carve-out
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, 85) != cudaSuccess)
+        return GRASS_ERR_CUDA;
     // sample chunks: enough CTAs for ~4 waves of the tiles on or above the diagonal, at least 256 samples each
     const int64_t tiles = (int64_t)d.tiles_m * (d.tiles_m + 1) / 2;
     int64_t want = (4 * (int64_t)sms * per_sm + tiles - 1) / tiles;
