@@ -61,6 +61,10 @@ def lib() -> ctypes.CDLL:
                                               vp, vp, vp, vp]
         L.oracle_score.restype = ctypes.c_int
         L.oracle_score.argtypes = [vp, i64, i64, vp, i64, i64, i64, vp, vp]
+        L.oracle_mask.restype = ctypes.c_int
+        L.oracle_mask.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, i64, vp]
+        L.oracle_factmask.restype = ctypes.c_int
+        L.oracle_factmask.argtypes = [vp, vp, ctypes.c_int, i32, i32, i32, i32, vp, i32, vp, i32, vp, vp]
         L.oracle_fim.restype = ctypes.c_int
         L.oracle_fim.argtypes = [vp, i64, i64, i64, vp, vp]
         L.oracle_fim_solve.restype = ctypes.c_int
@@ -185,6 +189,38 @@ def score(train: np.ndarray, test: np.ndarray, want_absum: bool = True):
     if rc:
         raise ValueError(f"oracle_score failed ({rc})")
     return sc, ab
+
+
+def mask(g: np.ndarray, idx, dtype: str = "f32", p=None) -> np.ndarray:
+    """Stand-alone Mask: out[i, j] = g[i, idx[j]] (float64)."""
+    _check_data(g, dtype)
+    n, ld = g.shape
+    p = ld if p is None else p
+    idx = np.ascontiguousarray(idx, dtype=np.uint32)
+    out = np.empty((n, idx.size), dtype=np.float64)
+    rc = lib().oracle_mask(_ptr(g), _DT[dtype], n, p, ld, _ptr(idx), idx.size, _ptr(out))
+    if rc:
+        raise ValueError(f"oracle_mask failed ({rc})")
+    return out
+
+
+def factmask(A: np.ndarray, G: np.ndarray, mask_in, mask_out, dtype: str = "bf16", want_absum: bool = True):
+    """Factorised Mask for one linear layer: the k'_in x k'_out block, flattened input-major."""
+    _check_data(A, dtype)
+    _check_data(G, dtype)
+    B, T, d_in = A.shape
+    d_out = G.shape[2]
+    assert G.shape[:2] == (B, T)
+    mask_in = np.ascontiguousarray(mask_in, dtype=np.uint32)
+    mask_out = np.ascontiguousarray(mask_out, dtype=np.uint32)
+    kp = mask_in.size * mask_out.size
+    out = np.empty((B, kp), dtype=np.float64)
+    ab = np.empty((B, kp), dtype=np.float64) if want_absum else None
+    rc = lib().oracle_factmask(_ptr(A), _ptr(G), _DT[dtype], B, T, d_in, d_out, _ptr(mask_in), mask_in.size,
+                               _ptr(mask_out), mask_out.size, _ptr(out), _ptr(ab))
+    if rc:
+        raise ValueError(f"oracle_factmask failed ({rc})")
+    return out, ab
 
 
 def fim(X: np.ndarray, want_absum: bool = True):

@@ -311,6 +311,49 @@ int oracle_score(const float *train, int64_t N, int64_t ld_train, const float *t
     return 0;
 }
 
+/* ---- stand-alone sparsification (Section 3.2; the paper evaluates Mask alone as a compressor) ----
+ * oracle_mask:     out[i, j] = g[i, idx[j]]                       (g-hat = M g, M the selection matrix)
+ * oracle_factmask: out[b, a*kout + c] = sum_t A[b,t,mask_in[a]] * G[b,t,mask_out[c]]
+ *                  (Mask_{k'_in (x) k'_out}: Eq. 2 with selection matrices, no projection afterwards)
+ * absum (factmask) is the same sum over absolute values. */
+int oracle_mask(const void *g, int dtype, int64_t n, int64_t p, int64_t ld, const uint32_t *idx,
+                int64_t kprime, double *out)
+{
+    if (kprime > p || ld < p) return 1;
+    for (int64_t i = 0; i < n; ++i)
+        for (int64_t j = 0; j < kprime; ++j) {
+            if ((int64_t)idx[j] >= p) return 1;
+            out[i * kprime + j] = load_elem(g, dtype, i * ld + idx[j]);
+        }
+    return 0;
+}
+
+int oracle_factmask(const void *A, const void *G, int dtype, int32_t B, int32_t T, int32_t d_in,
+                    int32_t d_out, const uint32_t *mask_in, int32_t kin, const uint32_t *mask_out,
+                    int32_t kout, double *out, double *absum)
+{
+    if (kin > d_in || kout > d_out) return 1;
+    const int64_t kp = (int64_t)kin * kout;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t b = 0; b < B; ++b) {
+        double *o = out + (int64_t)b * kp;
+        double *ab = absum ? absum + (int64_t)b * kp : NULL;
+        for (int64_t q = 0; q < kp; ++q) { o[q] = 0.0; if (ab) ab[q] = 0.0; }
+        for (int32_t t = 0; t < T; ++t) {
+            const int64_t row = (int64_t)b * T + t;
+            for (int32_t a = 0; a < kin; ++a) {
+                const double x = load_elem(A, dtype, row * d_in + mask_in[a]);
+                for (int32_t c = 0; c < kout; ++c) {
+                    const double y = load_elem(G, dtype, row * d_out + mask_out[c]);
+                    o[(int64_t)a * kout + c] += x * y;
+                    if (ab) ab[(int64_t)a * kout + c] += fabs(x * y);
+                }
+            }
+        }
+    }
+    return 0;
+}
+
 /* ---- projected Fisher information matrix and iFVP (Section 2.1, cache stage) ---
  * F = (1/n) sum_i g_i g_i^T over the n compressed gradients (rows of X, n x k,
  * row stride ld); with the layer-wise block-diagonal approximation of Section
