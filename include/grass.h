@@ -122,6 +122,27 @@ grass_status factgrass_compress_grouped(const factgrass_layer* layers /*host*/, 
 size_t factgrass_grouped_workspace_bytes(int32_t L);
 
 /*
+ * Sparsification alone (Section 3.2: Random / Selective Mask used as the whole compressor, which the
+ * paper evaluates next to GraSS and FactGraSS).
+ *   grass_mask         out[i, j] = g[i, idx[j]],  out n x kprime fp32 (row stride ld_out >= kprime);
+ *                      g and idx as in grass_compress (idx must not be NULL; n <= 65,535 per call).
+ *   factmask_compress  out[b, a*kout + c] = sum_t A[b,t,mask_in[a]] * G[b,t,mask_out[c]]: the k'_in x k'_out
+ *                      block of Eq. 2 with selection matrices, flattened input-major, without projection.
+ *                      out is B x (kin*kout) fp32; arguments as in factgrass_compress.
+ *   factmask_compress_grouped  the same for L layers; layer l writes out[b, out_offset .. + kin*kout);
+ *                      the `spec` member of the descriptors is ignored.
+ * An index >= the row length gives 0 in grass_mask (and is skipped in factmask) and sets GRASS_DEV_BAD_INDEX.
+ */
+grass_status grass_mask(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld, const uint32_t* idx,
+                        int64_t kprime, float* out, int64_t ld_out, uint32_t* dev_status, void* stream);
+grass_status factmask_compress(const void* A, const void* G, grass_dtype dt, int32_t B, int32_t T, int32_t d_in,
+                               int32_t d_out, const uint32_t* mask_in, int32_t kin, const uint32_t* mask_out,
+                               int32_t kout, float* out, int64_t ld_out, uint32_t* dev_status, void* stream);
+grass_status factmask_compress_grouped(const factgrass_layer* layers /*host*/, int32_t L, grass_dtype dt, int32_t B,
+                                       int32_t T, float* out, int64_t ld_out, void* workspace,
+                                       size_t workspace_bytes, uint32_t* dev_status, void* stream);
+
+/*
  * FactGraSS on batches whose samples have their own sequence lengths.  The sum over tokens in Eq. 2
  * (Section 3.3.2) runs over the tokens of one sample; padding tokens are not part of it, so they are
  * not read at all.  A and G of every layer are token-major matrices (rows x d_in, rows x d_out); the

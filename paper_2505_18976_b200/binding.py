@@ -25,7 +25,8 @@ DEV_BAD_INDEX, DEV_TIMEOUT, DEV_BAD_LENGTH, DEV_NOT_PD = 1, 2, 4, 8
 
 EXPORTS = ("grass_compress", "factgrass_compress", "factgrass_compress_grouped",
            "factgrass_compress_varlen", "factgrass_compress_grouped_varlen",
-           "grass_fim", "grass_fim_factor", "grass_fim_apply",
+           "grass_fim", "grass_fim_factor", "grass_fim_apply", "grass_mask", "factmask_compress",
+           "factmask_compress_grouped",
            "factgrass_grouped_workspace_bytes", "factgrass_compress_grouped_static", "grass_score", "grass_sjlt_table", "grass_validate_mask",
            "grass_random_mask_host", "grass_status_string")
 
@@ -80,6 +81,13 @@ def lib() -> ctypes.CDLL:
                                                         i64, vp, vp]
         L.grass_score.restype = st
         L.grass_score.argtypes = [vp, i64, i64, vp, i64, i64, i64, vp, i64, vp]
+        L.grass_mask.restype = st
+        L.grass_mask.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, i64, vp, i64, vp, vp]
+        L.factmask_compress.restype = st
+        L.factmask_compress.argtypes = [vp, vp, ctypes.c_int, i32, i32, i32, i32, vp, i32, vp, i32, vp, i64, vp, vp]
+        L.factmask_compress_grouped.restype = st
+        L.factmask_compress_grouped.argtypes = [ctypes.POINTER(FactgrassLayer), i32, ctypes.c_int, i32, i32, vp, i64,
+                                                vp, ctypes.c_size_t, vp, vp]
         L.grass_fim.restype = st
         L.grass_fim.argtypes = [vp, i64, i64, i64, vp, i64, vp]
         L.grass_fim_factor.restype = st
@@ -285,6 +293,50 @@ def grass_score(train: torch.Tensor, test: torch.Tensor, out: Optional[torch.Ten
     _check(lib().grass_score(_ptr(train), N, train.stride(0) if N > 1 else D, _ptr(test), M,
                              test.stride(0) if M > 1 else D, D, _ptr(out), out.stride(0) if N > 1 else M,
                              _stream()), "grass_score")
+    return out
+
+
+def grass_mask(g: torch.Tensor, idx: torch.Tensor, out: Optional[torch.Tensor] = None, p: Optional[int] = None,
+               dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Stand-alone Mask: out[i, j] = g[i, idx[j]] as fp32."""
+    _need_cuda(g, idx, out, dev_status)
+    assert g.dim() == 2 and g.stride(1) == 1
+    n, ld = g.shape[0], g.stride(0) if g.shape[0] > 1 else g.shape[1]
+    p = g.shape[1] if p is None else p
+    kp = idx.numel()
+    if out is None:
+        out = torch.empty((n, kp), dtype=torch.float32, device=g.device)
+    _check(lib().grass_mask(_ptr(g), _dt(g), n, p, ld, _ptr(idx), kp, _ptr(out),
+                            out.stride(0) if n > 1 else max(out.shape[1], kp), _ptr(dev_status), _stream()), "grass_mask")
+    return out
+
+
+def factmask_compress(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, mask_out: torch.Tensor,
+                      out: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Factorised Mask of one linear layer: out[b, a*kout + c] = sum_t A[b,t,mask_in[a]] G[b,t,mask_out[c]]."""
+    _need_cuda(A, G, mask_in, mask_out, out, dev_status)
+    assert A.is_contiguous() and G.is_contiguous() and A.dim() == 3 and G.dim() == 3 and A.dtype == G.dtype
+    B, T, d_in = A.shape
+    d_out = G.shape[2]
+    kp = mask_in.numel() * mask_out.numel()
+    if out is None:
+        out = torch.empty((B, kp), dtype=torch.float32, device=A.device)
+    _check(lib().factmask_compress(_ptr(A), _ptr(G), _dt(A), B, T, d_in, d_out, _ptr(mask_in), mask_in.numel(),
+                                   _ptr(mask_out), mask_out.numel(), _ptr(out),
+                                   out.stride(0) if B > 1 else max(out.shape[1], kp), _ptr(dev_status), _stream()),
+           "factmask_compress")
+    return out
+
+
+def factmask_compress_grouped(group: "GroupedLayers", out: torch.Tensor, workspace: torch.Tensor,
+                              dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Factorised Mask of all layers of ``group`` in one launch (the layers' k, s, seed are ignored)."""
+    _need_cuda(out, workspace, dev_status)
+    assert out.dtype == torch.float32 and out.stride(1) == 1
+    _check(lib().factmask_compress_grouped(group.array, group.L, group.dtype, group.B, group.T, _ptr(out),
+                                           out.stride(0) if out.shape[0] > 1 else out.shape[1], _ptr(workspace),
+                                           workspace.numel() * workspace.element_size(), _ptr(dev_status),
+                                           _stream()), "factmask_compress_grouped")
     return out
 
 

@@ -18,6 +18,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 namespace grass {
 
@@ -55,6 +56,7 @@ __device__ __forceinline__ uint4 pack8_bf16(const uint32_t (&v)[8])
 
 // What happens to the finished k'_in x k'_out block.
 constexpr int kEpiSjlt = 0;   // FactGraSS stage 3: hash every entry into the k-bin accumulator
+constexpr int kEpiBlock = 2;  // factorised Mask alone (Section 3.2): add the block itself into out[b, off + a*kout + c]
 constexpr int kEpiRaw = 1;    // add scale * block into a dense symmetric matrix (projected FIM, see grass_fim.cu):
                               // only tiles on or above the diagonal are computed, the others are mirrored
 
@@ -249,7 +251,9 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     const int quarter = warp & 3;
     const uint32_t tq = tmem_d + ((uint32_t)(quarter * 32) << 16);
     auto project = [&](int a, int c, float val) {
-        if constexpr (EPI == kEpiRaw) {
+        if constexpr (EPI == kEpiBlock) {
+            if (a < kin && c < kout && val != 0.0f) atomicAdd(orow + (int64_t)a * kout + c, val);
+        } else if constexpr (EPI == kEpiRaw) {
             // tiles above the diagonal fill their mirror image too; a diagonal tile uses its upper half
             if (a < kin && c < kout && (tm != tn || a <= c)) {
                 const float sv = val * L.scale;
@@ -368,7 +372,8 @@ static int fg_env_int(const char* name, int dflt)
 
 static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, grass_dtype dt, int32_t B, int32_t T,
                                   const int64_t* tok_begin, const int32_t* tok_count, float* out, int64_t ld_out,
-                                  void* workspace, size_t workspace_bytes, uint32_t* dev_status, cudaStream_t st)
+                                  void* workspace, size_t workspace_bytes, uint32_t* dev_status, cudaStream_t st,
+                                  int epi = kEpiSjlt)
 {
     if (L < 0 || B < 0 || T < 0 || (L > 0 && !layers)) return GRASS_ERR_INVALID_ARG;
     if (dt != GRASS_BF16 && dt != GRASS_F32) return GRASS_ERR_INVALID_ARG;
@@ -433,7 +438,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
 
-    const size_t bins_bytes = (size_t)max_k_smem * sizeof(float);
+    const size_t bins_bytes = epi == kEpiSjlt ? (size_t)max_k_smem * sizeof(float) : 0;
     const bool f32 = dt == GRASS_F32;
     auto launch = [&](auto kern, size_t stage_bytes) -> grass_status {
         const size_t smem = 2 * stage_bytes + bins_bytes;
@@ -492,11 +497,36 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
         return launch_status();
     };
     const size_t piece = (size_t)tile * tc::ROW_BYTES * 2;   // one bf16 piece of the A tile plus one of the G tile
+    if (epi == kEpiBlock) {
+        if (tile == 64)
+            return f32 ? launch(factgrass_kernel<64, 64, true, kEpiBlock>, 3 * piece)
+                       : launch(factgrass_kernel<64, 64, false, kEpiBlock>, piece);
+        return f32 ? launch(factgrass_kernel<128, 128, true, kEpiBlock>, 3 * piece)
+                   : launch(factgrass_kernel<128, 128, false, kEpiBlock>, piece);
+    }
     if (tile == 64)
         return f32 ? launch(factgrass_kernel<64, 64, true, kEpiSjlt>, 3 * piece)
                    : launch(factgrass_kernel<64, 64, false, kEpiSjlt>, piece);
     return f32 ? launch(factgrass_kernel<128, 128, true, kEpiSjlt>, 3 * piece)
                : launch(factgrass_kernel<128, 128, false, kEpiSjlt>, piece);
+}
+
+// Factorised Mask without projection: the layers' specs are replaced by k = kin * kout (the block itself
+// is the output) and the kernels run with the block epilogue.
+static grass_status run_factmask(const factgrass_layer* layers, int32_t L, grass_dtype dt, int32_t B, int32_t T,
+                                 float* out, int64_t ld_out, void* workspace, size_t workspace_bytes,
+                                 uint32_t* dev_status, cudaStream_t st)
+{
+    if (L < 0 || (L > 0 && !layers)) return GRASS_ERR_INVALID_ARG;
+    std::vector<factgrass_layer> tmp(layers, layers + L);
+    for (auto& l : tmp) {
+        if (l.kin < 0 || l.kout < 0 || (int64_t)l.kin * l.kout > 0x7FFFFFFFLL) return GRASS_ERR_INVALID_ARG;
+        l.spec.k = (uint32_t)std::max<int64_t>((int64_t)l.kin * l.kout, 1);
+        l.spec.s = 1;
+        l.spec.seed = 0;
+    }
+    return run_factgrass(tmp.data(), L, dt, B, T, nullptr, nullptr, out, ld_out, workspace, workspace_bytes, dev_status,
+                         st, kEpiBlock);
 }
 
 // Projected Fisher information matrix F = scale * X^T X of the n rows of X (n x k fp32, row stride ld):
@@ -584,6 +614,36 @@ extern "C" grass_status factgrass_compress_varlen(const void* A, const void* G, 
     l.out_offset = 0;
     return grass::run_factgrass(&l, 1, dt, B, T_max, tok_begin, tok_count, out, ld_out, nullptr, 0, dev_status,
                                 (cudaStream_t)stream);
+}
+
+extern "C" grass_status factmask_compress(const void* A, const void* G, grass_dtype dt, int32_t B, int32_t T,
+                                          int32_t d_in, int32_t d_out, const uint32_t* mask_in, int32_t kin,
+                                          const uint32_t* mask_out, int32_t kout, float* out, int64_t ld_out,
+                                          uint32_t* dev_status, void* stream)
+{
+    factgrass_layer l;
+    l.A = A;
+    l.G = G;
+    l.mask_in = mask_in;
+    l.mask_out = mask_out;
+    l.d_in = d_in;
+    l.d_out = d_out;
+    l.kin = kin;
+    l.kout = kout;
+    l.spec.k = 1;
+    l.spec.s = 1;
+    l.spec.seed = 0;
+    l.out_offset = 0;
+    return grass::run_factmask(&l, 1, dt, B, T, out, ld_out, nullptr, 0, dev_status, (cudaStream_t)stream);
+}
+
+extern "C" grass_status factmask_compress_grouped(const factgrass_layer* layers, int32_t L, grass_dtype dt, int32_t B,
+                                                  int32_t T, float* out, int64_t ld_out, void* workspace,
+                                                  size_t workspace_bytes, uint32_t* dev_status, void* stream)
+{
+    if (!workspace) return GRASS_ERR_INVALID_ARG;
+    return grass::run_factmask(layers, L, dt, B, T, out, ld_out, workspace, workspace_bytes, dev_status,
+                               (cudaStream_t)stream);
 }
 
 extern "C" size_t factgrass_grouped_workspace_bytes(int32_t L)

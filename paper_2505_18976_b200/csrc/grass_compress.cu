@@ -119,6 +119,25 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
     }
 }
 
+// Stand-alone Mask_k' (Section 3.2): out[i, j] = g[i, idx[j]], written as fp32.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+grass_mask_kernel(const T* __restrict__ g, int64_t p, int64_t ld, const uint32_t* __restrict__ idx, int64_t kprime,
+                  float* __restrict__ out, int64_t ld_out, uint32_t* dev_status)
+{
+    const int64_t i = blockIdx.y;
+    const T* row = g + i * ld;
+    float* orow = out + i * ld_out;
+    bool bad = false;
+    for (int64_t j = (int64_t)blockIdx.x * kThreads * 4 + threadIdx.x; j < kprime && j < ((int64_t)blockIdx.x + 1) * kThreads * 4;
+         j += kThreads) {
+        const uint32_t c = __ldg(idx + j);
+        if ((int64_t)c >= p) { bad = true; orow[j] = 0.0f; continue; }
+        orow[j] = elem<T>::load(row + c);
+    }
+    if (bad && dev_status) atomicOr(dev_status, GRASS_DEV_BAD_INDEX);
+}
+
 struct CompressPlan {
     int S;          // samples per CTA
     int jsplit;     // CTAs that share one sample group (split of the masked positions)
@@ -232,6 +251,25 @@ static grass_status dispatch_compress(const T* g, int64_t n, int64_t p, int64_t 
 }
 
 }  // namespace grass
+
+extern "C" grass_status grass_mask(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld, const uint32_t* idx,
+                                   int64_t kprime, float* out, int64_t ld_out, uint32_t* dev_status, void* stream)
+{
+    if (n < 0 || p < 0 || kprime < 0 || kprime > p || ld < p || ld_out < kprime) return GRASS_ERR_INVALID_ARG;
+    if (p >= 0xFFFFFFFFLL || n > 65535) return n > 65535 ? GRASS_ERR_UNSUPPORTED : GRASS_ERR_INVALID_ARG;
+    if (dt != GRASS_F32 && dt != GRASS_BF16) return GRASS_ERR_UNSUPPORTED;
+    if (n == 0 || kprime == 0) return GRASS_OK;
+    if (!g || !idx || !out) return GRASS_ERR_INVALID_ARG;
+    dim3 grid((unsigned)((kprime + grass::kThreads * 4 - 1) / (grass::kThreads * 4)), (unsigned)n);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (dt == GRASS_F32)
+        grass::grass_mask_kernel<float><<<grid, grass::kThreads, 0, st>>>((const float*)g, p, ld, idx, kprime, out, ld_out,
+                                                                          dev_status);
+    else
+        grass::grass_mask_kernel<__nv_bfloat16><<<grid, grass::kThreads, 0, st>>>((const __nv_bfloat16*)g, p, ld, idx,
+                                                                                  kprime, out, ld_out, dev_status);
+    return grass::launch_status();
+}
 
 extern "C" grass_status grass_compress(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld,
                                        const uint32_t* idx, int64_t kprime, const grass_sjlt_spec* spec,
