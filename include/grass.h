@@ -219,7 +219,8 @@ grass_status grass_fim(const float* X, int64_t n, int64_t k, int64_t ld, float* 
  * Damped inverse-FIM-vector products (Section 2.1, cache stage step 3: g~ = F^-1 g; the damping term
  * lambda is the hyper-parameter of the paper's appendix on experiment details).
  *   grass_fim_factor  replaces the lower triangle of F by the Cholesky factor L of F + lambda*I
- *                     (lambda >= 0; the strict upper triangle is left as it was and is not used again).
+ *                     (lambda >= 0; the strict upper triangle is scratch: the 64 x 64 diagonal blocks keep the
+ *                     inverses of their factors there, the rest is left as it was).
  *                     If a pivot is not positive, GRASS_DEV_NOT_PD is OR-ed into *dev_status (nullable)
  *                     and the result is meaningless; nothing traps.
  *   grass_fim_apply   overwrites each of the M rows b_m of Bm (M x k fp32, row stride ld_b >= k) by

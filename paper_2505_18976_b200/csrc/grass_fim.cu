@@ -3,7 +3,8 @@
 //
 //   grass_fim         F = (1/n) sum_i g_i g_i^T over compressed gradients: the tensor-core contraction of
 //                     the FactGraSS kernel with both factors equal to the gradient matrix (factgrass.cu).
-//   grass_fim_factor  F + lambda I = L L^T, blocked right-looking Cholesky in fp32, in place (lower part).
+//   grass_fim_factor  F + lambda I = L L^T, blocked right-looking Cholesky in fp32, in place (lower part;
+//                     the diagonal blocks' upper triangles receive the inverses of the diagonal factors).
 //   grass_fim_apply   rows b_m <- (L L^T)^-1 b_m by blocked forward and back substitution.
 //
 // The factorisation and the substitutions are plain fp32 FMA kernels on 64-wide blocks: a diagonal-block
@@ -26,19 +27,38 @@ __global__ void add_damping_kernel(float* __restrict__ F, int64_t k, int64_t ld,
     if (i < k) F[i * ld + i] += lambda;
 }
 
-// Unblocked Cholesky of the jb x jb diagonal block at (j0, j0), one CTA.  A pivot that is not positive
-// sets GRASS_DEV_NOT_PD and is replaced by 1 so that nothing divides by zero.
+// Unblocked Cholesky of the jb x jb diagonal block at (j0, j0), one CTA, followed by the inverse of the
+// triangular factor.  On return the block's lower triangle holds Ljj and its strict upper triangle holds the
+// strict lower triangle of Ljj^-1, transposed (the diagonal of the inverse is 1 / diag(Ljj)): the upper
+// triangle of F is not used by anything else, and with the inverse at hand every triangular solve against
+// this block becomes a small matrix product.  A pivot that is not positive sets GRASS_DEV_NOT_PD and is
+// replaced by 1 so that nothing divides by zero.
 __global__ void __launch_bounds__(256)
 potrf_diag_kernel(float* __restrict__ F, int64_t ld, int64_t j0, int jb, uint32_t* dev_status)
 {
     __shared__ float a[NB][NB + 1];
+    __shared__ float inv[NB][NB + 1];
     const int tid = threadIdx.x;
     float* blk = F + j0 * ld + j0;
-    for (int e = tid; e < jb * jb; e += 256) {
-        const int i = e / jb, j = e % jb;
-        a[i][j] = (j <= i) ? blk[(int64_t)i * ld + j] : 0.0f;
+    // rows and columns beyond jb are padded with the identity, so the loops below have fixed bounds
+    {
+        float v[NB * NB / 256];
+#pragma unroll
+        for (int u = 0; u < NB * NB / 256; ++u) {
+            const int e = tid + u * 256, r = e / NB, c = e % NB;
+            v[u] = (r < jb && c <= r) ? blk[(int64_t)r * ld + c] : ((r == c && r >= jb) ? 1.0f : 0.0f);
+        }
+#pragma unroll
+        for (int u = 0; u < NB * NB / 256; ++u) {
+            const int e = tid + u * 256;
+            a[e / NB][e % NB] = v[u];
+            inv[e / NB][e % NB] = 0.0f;
+        }
     }
-    for (int c = 0; c < jb; ++c) {
+    // thread (i, jq) owns row i, columns jq, jq + 4, ..., jq + 60
+    const int i = tid >> 2, jq = tid & 3;
+#pragma unroll 1
+    for (int c = 0; c < NB; ++c) {
         __syncthreads();
         float d = a[c][c];
         if (!(d > 0.0f)) {
@@ -47,64 +67,108 @@ potrf_diag_kernel(float* __restrict__ F, int64_t ld, int64_t j0, int jb, uint32_
         }
         const float sd = sqrtf(d);
         __syncthreads();
-        if (tid < jb - c) {
-            const int i = c + tid;
-            a[i][c] = (i == c) ? sd : a[i][c] / sd;
-        }
+        if (jq == 0 && i >= c) a[i][c] = (i == c) ? sd : a[i][c] / sd;
         __syncthreads();
-        const int m = jb - c - 1;
-        for (int e = tid; e < m * m; e += 256) {
-            const int i = c + 1 + e / m, j = c + 1 + e % m;
-            if (j <= i) a[i][j] -= a[i][c] * a[j][c];
+        if (i > c) {
+            const float lic = a[i][c];
+            float t[NB / 4], l[NB / 4];
+#pragma unroll
+            for (int m = 0; m < NB / 4; ++m) {           // all loads first: they are independent
+                t[m] = a[i][jq + 4 * m];
+                l[m] = a[jq + 4 * m][c];
+            }
+#pragma unroll
+            for (int m = 0; m < NB / 4; ++m) {
+                const int j = jq + 4 * m;
+                if (j > c && j <= i) a[i][j] = fmaf(-lic, l[m], t[m]);
+            }
         }
     }
     __syncthreads();
-    for (int e = tid; e < jb * jb; e += 256) {
-        const int i = e / jb, j = e % jb;
-        if (j <= i) blk[(int64_t)i * ld + j] = a[i][j];
+    // inverse of the factor by forward substitution: a quad of lanes per column, each lane summing every
+    // fourth term; all lanes run the same number of steps because the shuffles are warp-wide
+    {
+        const int col = tid >> 2, part = tid & 3;
+#pragma unroll 1
+        for (int r = 0; r < NB; ++r) {
+            float fa[NB / 4], fx[NB / 4];
+#pragma unroll
+            for (int m = 0; m < NB / 4; ++m) {
+                fa[m] = a[r][part + 4 * m];
+                fx[m] = inv[part + 4 * m][col];          // zero above the diagonal and where not yet computed
+            }
+            float v = 0.0f;
+#pragma unroll
+            for (int m = 0; m < NB / 4; ++m)
+                if (part + 4 * m < r) v = fmaf(-fa[m], fx[m], v);
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+            if (part == 0 && r >= col) inv[r][col] = ((r == col ? 1.0f : 0.0f) + v) / a[r][r];
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < NB * NB / 256; ++u) {
+        const int e = tid + u * 256, r = e / NB, c = e % NB;
+        if (r < jb && c < jb) blk[(int64_t)r * ld + c] = (c <= r) ? a[r][c] : inv[c][r];
     }
 }
 
-// Rows r of C (rows x jb, at column offset of the block) solved against the diagonal block Ljj (jb x jb,
-// lower):  forward  x Ljj^T = c  (x[q] = (c[q] - sum_{p<q} x[p] L[q][p]) / L[q][q]),
-//          backward x Ljj   = c  (x[q] = (c[q] - sum_{p>q} x[p] L[p][q]) / L[q][q]).
-// One thread per row for the substitution, 64 rows per CTA; all 256 threads move the data.
+// Rows of C (rows x jb, at the block's column offset) solved against the diagonal block through its stored
+// inverse (see potrf_diag_kernel):  forward  x Ljj^T = c  ->  x = c (Ljj^-1)^T,   backward  x Ljj = c  ->
+// x = c Ljj^-1.  64 rows per CTA, a 4 x 4 register tile of the product per thread.
 template <bool BACKWARD>
 __global__ void __launch_bounds__(256)
 trsm_rows_kernel(const float* __restrict__ Ljj, int64_t ld_l, int jb, float* __restrict__ C, int64_t ld_c, int64_t rows)
 {
-    __shared__ float l[NB][NB + 1];
-    __shared__ float x[NB][NB + 1];   // x[q][r]
+    __shared__ __align__(16) float w[NB][NB + 4];    // w[p][q]: x[q] = sum_p c[p] * w[p][q]
+    __shared__ __align__(16) float ct[NB][NB + 4];   // ct[p][r] = c[r][p]
     const int tid = threadIdx.x;
     const int64_t r0 = (int64_t)blockIdx.x * NB;
-#pragma unroll 4
-    for (int e = tid; e < NB * NB; e += 256) {
-        const int i = e / NB, j = e % NB;             // consecutive threads read consecutive columns
-        l[i][j] = (i < jb && j <= i) ? Ljj[(int64_t)i * ld_l + j] : 0.0f;
-        x[j][i] = (j < jb && r0 + i < rows) ? C[(r0 + i) * ld_c + j] : 0.0f;
+    float lraw[NB * NB / 256], craw[NB * NB / 256];
+#pragma unroll
+    for (int u = 0; u < NB * NB / 256; ++u) {        // all global loads first: they are independent
+        const int e = tid + u * 256, i = e / NB, j = e % NB;
+        lraw[u] = (i < jb && j < jb) ? Ljj[(int64_t)i * ld_l + j] : 0.0f;
+        craw[u] = (j < jb && r0 + i < rows) ? C[(r0 + i) * ld_c + j] : 0.0f;
+    }
+#pragma unroll
+    for (int u = 0; u < NB * NB / 256; ++u) {
+        const int e = tid + u * 256, i = e / NB, j = e % NB;   // consecutive threads: consecutive columns
+        float v = 0.0f;
+        if (i < jb && j < jb) v = (i == j) ? 1.0f / lraw[u] : lraw[u];   // j > i: inverse entry (j, i); j < i: unused
+        // inverse entry (row a, col b), a >= b, is stored at block position [b][a]
+        if (!BACKWARD) { w[i][j] = (j >= i) ? v : 0.0f; }                        // w[p][q] = inv[q][p], p <= q
+        else           { if (j >= i) w[j][i] = v; if (j > i) w[i][j] = 0.0f; }   // w[p][q] = inv[p][q], p >= q
+        ct[j][i] = craw[u];
     }
     __syncthreads();
-    if (tid < NB) {
-        const int r = tid;
-        if (!BACKWARD) {
-            for (int q = 0; q < jb; ++q) {
-                float v = x[q][r];
-                for (int p = 0; p < q; ++p) v = fmaf(-x[p][r], l[q][p], v);
-                x[q][r] = v / l[q][q];
-            }
-        } else {
-            for (int q = jb - 1; q >= 0; --q) {
-                float v = x[q][r];
-                for (int p = q + 1; p < jb; ++p) v = fmaf(-x[p][r], l[p][q], v);
-                x[q][r] = v / l[q][q];
-            }
+    const int ty = tid / 16, tx = tid % 16;          // rows ty*4.., outputs tx*4..
+    float acc[4][4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) acc[u][v] = 0.0f;
+#pragma unroll 8
+    for (int p = 0; p < NB; ++p) {
+        const float4 c4 = *reinterpret_cast<const float4*>(&ct[p][ty * 4]);
+        const float4 w4 = *reinterpret_cast<const float4*>(&w[p][tx * 4]);
+        const float c[4] = {c4.x, c4.y, c4.z, c4.w}, ww[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) acc[u][v] = fmaf(c[u], ww[v], acc[u][v]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int64_t r = r0 + ty * 4 + u;
+        if (r >= rows) continue;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int q = tx * 4 + v;
+            if (q < jb) C[r * ld_c + q] = acc[u][v];
         }
-    }
-    __syncthreads();
-#pragma unroll 4
-    for (int e = tid; e < NB * NB; e += 256) {
-        const int i = e / NB, j = e % NB;
-        if (j < jb && r0 + i < rows) C[(r0 + i) * ld_c + j] = x[j][i];
     }
 }
 
@@ -121,16 +185,22 @@ gemm_sub_kernel(float* __restrict__ C, int64_t ldc, int64_t rows, int64_t cols, 
     __shared__ __align__(16) float bs[NB][NB + 4];   // bs[q][j]
     const int tid = threadIdx.x;
     const int64_t i0 = (int64_t)blockIdx.y * NB, j0 = (int64_t)blockIdx.x * NB;
-    for (int e = tid; e < NB * NB; e += 256) {
-        const int rr = e / NB, q = e % NB;            // consecutive threads read consecutive q of one row
-        as[q][rr] = (i0 + rr < rows && q < K) ? A[(i0 + rr) * lda + q] : 0.0f;
-        if (!B_TRANS) bs[q][rr] = (j0 + rr < cols && q < K) ? Bm[(j0 + rr) * ldb + q] : 0.0f;
-    }
-    if (B_TRANS)
-        for (int e = tid; e < NB * NB; e += 256) {
-            const int q = e / NB, jj = e % NB;        // consecutive threads read consecutive j of one q
-            bs[q][jj] = (j0 + jj < cols && q < K) ? Bm[(int64_t)q * ldb + j0 + jj] : 0.0f;
+    {
+        float av[NB * NB / 256], bv[NB * NB / 256];
+#pragma unroll
+        for (int u = 0; u < NB * NB / 256; ++u) {     // all global loads first: they are independent
+            const int e = tid + u * 256, hi = e / NB, lo = e % NB;   // consecutive threads: consecutive addresses
+            av[u] = (i0 + hi < rows && lo < K) ? A[(i0 + hi) * lda + lo] : 0.0f;
+            if (!B_TRANS) bv[u] = (j0 + hi < cols && lo < K) ? Bm[(j0 + hi) * ldb + lo] : 0.0f;
+            else bv[u] = (j0 + lo < cols && hi < K) ? Bm[(int64_t)hi * ldb + j0 + lo] : 0.0f;
         }
+#pragma unroll
+        for (int u = 0; u < NB * NB / 256; ++u) {
+            const int e = tid + u * 256, hi = e / NB, lo = e % NB;
+            as[lo][hi] = av[u];
+            if (!B_TRANS) bs[lo][hi] = bv[u]; else bs[hi][lo] = bv[u];
+        }
+    }
     __syncthreads();
     const int ty = tid / 16, tx = tid % 16;
     float acc[4][4];
