@@ -39,7 +39,7 @@ constexpr int A_SPLIT_BYTES = BM * BK * 2;   // one bf16 piece of the train tile
 constexpr int B_SPLIT_BYTES = BN * BK * 2;   // one bf16 piece of the test tile:  16 KB
 constexpr int STAGE_BYTES = 3 * (A_SPLIT_BYTES + B_SPLIT_BYTES);   // 72 KB
 constexpr int CHUNKS = BK / 8;     // 16-byte chunks (8 bf16) per row per stage
-constexpr int TASKS = (BM + BN) * CHUNKS / PRODUCERS;   // (row, chunk) tasks per producer per stage = 6
+constexpr int TASKS = (BM + BN) * CHUNKS / PRODUCERS;   // (row, chunk) tasks per producer per stage (3 with 16 producer warps)
 constexpr uint32_t TMEM_COLS = 512;   // two fp32 accumulators of BN columns each
 __global__ void __launch_bounds__(THREADS, 1)
 grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_train, const float* __restrict__ test,
