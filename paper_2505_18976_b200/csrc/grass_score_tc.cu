@@ -1,4 +1,4 @@
-// grass_score on the 5th-generation tensor cores (tcgen05 + TMEM), fp32-accurate.
+// grass_score on the 5th-generation tensor cores (tcgen05 + TMEM), fp32-accurate, CTA pairs, TMA loads.
 //
 // scores[i, m] = <train[i, :], test[m, :]> (attribute stage, Section 2.1) is the one dense contraction
 // of the path.  fp32 inputs are split exactly into three bf16 pieces, x = hi + mid + lo (8 significant
@@ -7,108 +7,174 @@
 // below 2^-23 of |x||y|, the size of one fp32 rounding.  hi*hi accumulates in one fp32 tile in tensor
 // memory and the five correction terms in a second one; the epilogue adds the two.
 //
-// One CTA owns a 128 x (<=256) output tile: 128 train rows (MMA M) by up to 256 test rows (MMA N).
-//   producer warps: read fp32 rows from HBM (the next k tile in registers while the current one is split),
-//              split, and write the bf16 pieces into shared memory in the tensor core's K-major layout with
-//              the 64-byte swizzle (64-byte rows; conflict-free 16-byte stores); then drain the accumulators;
-//   last warp  one elected thread issues tcgen05.mma (M=128, N<=256, K=16) and commits stage-free and
-//              accumulator-ready mbarriers.
-// Three 72 KB stages of 32 k-values each.  Every mbarrier wait is bounded: if one expires the CTA marks
-// its tile with NaN, still frees its tensor memory, and returns.
+// Two CTAs on neighbouring SMs (a cluster of 2) own a 256 x (<=256) output tile and run one
+// tcgen05.mma.cta_group::2 (M = 256, N <= 256, K = 16) per product: each CTA stages its own 128 train
+// rows and HALF of the test rows, the tensor cores of both SMs read both halves, and each CTA ends up
+// with its 128 x N accumulators in its own tensor memory.
+//   warp 17    one thread brings the raw fp32 tiles (128 rows x 32 k-values each, train and test) from
+//              global memory into a ring of shared-memory slots with TMA (cp.async.bulk.tensor.2d, 128-byte
+//              swizzle, no multicast); rows and k-values beyond the matrices arrive as zeros;
+//   warps 0-15 producers: read a raw slot, split, and write the bf16 pieces into shared memory in the tensor
+//              core's K-major layout with the 64-byte swizzle; one lane per warp then arrives on the LEADER
+//              CTA's "full" barrier (a remote arrive for the second CTA) and frees the raw slot; afterwards
+//              they drain their own CTA's accumulators;
+//   warp 16    allocates / frees tensor memory in both CTAs; in the leader CTA one elected thread issues
+//              the MMAs and commits, multicast to both CTAs, the stage-free and accumulator-ready barriers.
+// Two 48 KB operand stages and three 32 KB raw slots of 32 k-values each.  Every mbarrier wait is bounded:
+// if one expires the CTA marks its tile with NaN, still frees its tensor memory, and returns; the cluster
+// barriers are reached by every thread of both CTAs unconditionally.
+// The TMA path needs 16-byte aligned bases and row strides; other inputs take the plain FMA kernel
+// (grass_score.cu).
+#include <cuda.h>
+
 #include "grass_common.cuh"
 #include "tcgen05_util.cuh"
 
 namespace grass {
 namespace tc {
 
-constexpr int BM = 128;            // train rows per CTA (MMA M)
-constexpr int BN = 256;            // test rows per CTA (MMA N, upper bound)
-constexpr int STAGES = 3;
-#ifndef GRASS_SCORE_PRODUCERS
-#define GRASS_SCORE_PRODUCERS 512
-#endif
-#ifndef GRASS_SCORE_PREFETCH
-#define GRASS_SCORE_PREFETCH 1
-#endif
-constexpr int PRODUCERS = GRASS_SCORE_PRODUCERS;   // threads of the producer warps
+constexpr int BM = 128;            // train rows per CTA (the pair's MMA M is 256)
+constexpr int BN = 256;            // test rows per CTA pair (MMA N, upper bound); each CTA stages half
+constexpr int BNH = BN / 2;
+constexpr int STAGES = 2;          // bf16 operand stages
+constexpr int RING = 3;            // raw fp32 slots filled by TMA
+constexpr int PRODUCERS = 512;     // threads of the producer warps
 constexpr int PWARPS = PRODUCERS / 32;
-constexpr int PF = GRASS_SCORE_PREFETCH;           // k tiles of global loads in flight ahead of the one being split
-constexpr int RING = PF + 1;
-constexpr int THREADS = PRODUCERS + 32;
-constexpr int A_SPLIT_BYTES = BM * BK * 2;   // one bf16 piece of the train tile:  8 KB
-constexpr int B_SPLIT_BYTES = BN * BK * 2;   // one bf16 piece of the test tile:  16 KB
-constexpr int STAGE_BYTES = 3 * (A_SPLIT_BYTES + B_SPLIT_BYTES);   // 72 KB
+constexpr int THREADS = PRODUCERS + 64;   // + the MMA / tensor-memory warp and the TMA warp
+constexpr int A_SPLIT_BYTES = BM * BK * 2;    // one bf16 piece of the train tile: 8 KB
+constexpr int B_SPLIT_BYTES = BNH * BK * 2;   // one bf16 piece of this CTA's half of the test tile: 8 KB
+constexpr int STAGE_BYTES = 3 * (A_SPLIT_BYTES + B_SPLIT_BYTES);   // 48 KB
 constexpr int CHUNKS = BK / 8;     // 16-byte chunks (8 bf16) per row per stage
-constexpr int TASKS = (BM + BN) * CHUNKS / PRODUCERS;   // (row, chunk) tasks per producer per stage (3 with 16 producer warps)
+constexpr int TASKS = (BM + BNH) * CHUNKS / PRODUCERS;   // (row, chunk) tasks per producer per stage = 2
 constexpr uint32_t TMEM_COLS = 512;   // two fp32 accumulators of BN columns each
-__global__ void __launch_bounds__(THREADS, 1)
-grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_train, const float* __restrict__ test,
-                      int64_t M, int64_t ld_test, int64_t D, float* __restrict__ scores, int64_t ld_s, int vec_ok,
-                      int out_vec_ok)
+constexpr int RAW_HALF = BM * BK * 4;            // one raw fp32 tile (128 rows x 32 k-values): 16 KB
+constexpr int RAW_BYTES = 2 * RAW_HALF;          // train tile + this CTA's test tile
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + RING * RAW_BYTES;
+static_assert(BM == BNH, "both raw tiles use the same TMA box");
+static_assert(SMEM_BYTES <= 224 * 1024 && STAGE_BYTES % 1024 == 0 && RAW_HALF % 1024 == 0, "shared memory layout");
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// 2-D tiled TMA load into this CTA's shared memory; x = first k-value (a multiple of 32: 128 bytes), y = first row
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    return ra;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// bounded wait with cluster-scope acquire (the arrivals come from both CTAs)
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred P;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, P;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrives on the barrier at this shared-memory offset in both CTAs once all MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask)
+                 : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __grid_constant__ CUtensorMap map_test,
+                      int64_t N, int64_t M, int64_t D, float* __restrict__ scores, int64_t ld_s, int out_vec_ok)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
-    __shared__ __align__(8) unsigned long long bars[2 * STAGES + 1];
+    __shared__ __align__(8) unsigned long long bars[2 * STAGES + 1 + 2 * RING];
     __shared__ uint32_t tmem_base_slot;
     __shared__ volatile int abort_flag;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int64_t n0 = (int64_t)blockIdx.x * BM;
+    const uint32_t rank = cluster_ctarank();                       // 0 = leader (issues the MMAs)
+    const int64_t n0 = (int64_t)blockIdx.x * BM;                   // this CTA's train rows
     const int64_t m0 = (int64_t)blockIdx.y * BN;
-    const int64_t m_rows = (M - m0) < BN ? (M - m0) : BN;          // test rows of this tile
-    const uint32_t n_mma = (uint32_t)((m_rows + 15) / 16 * 16);    // MMA N (multiple of 16 for M = 128)
+    const int64_t m_rows = (M - m0) < BN ? (M - m0) : BN;          // test rows of the pair's tile
+    const uint32_t n_mma = (uint32_t)((m_rows + 15) / 16 * 16);    // MMA N (a multiple of 16 for M = 256)
+    const int n_half = (int)(n_mma / 2);                           // test rows staged by each CTA
     const int64_t ktiles = (D + BK - 1) / BK;
 
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), accum = smem_u32(&bars[2 * STAGES]);
+    const uint32_t rawfull0 = smem_u32(&bars[2 * STAGES + 1]), rawempty0 = rawfull0 + 8 * RING;
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full0 + 8 * s, PRODUCERS);
+            mbar_init(full0 + 8 * s, 2 * PWARPS);   // one arrival per producer warp of both CTAs (used in the leader)
             mbar_init(empty0 + 8 * s, 1);
         }
         mbar_init(accum, 1);
+        for (int r = 0; r < RING; ++r) {
+            mbar_init(rawfull0 + 8 * r, 1);        // the TMA thread's expect_tx arrival + the bytes
+            mbar_init(rawempty0 + 8 * r, PWARPS);  // one arrival per producer warp
+        }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == PWARPS) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                      "r"(TMEM_COLS)
                      : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    cluster_sync_all();            // both CTAs' barriers are initialised before anybody arrives remotely
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_d = tmem_base_slot;
     const uint32_t smem_base = smem_u32(smem);
 
     if (warp < PWARPS) {
         // ---------------- producers ----------------
-        // task q of this thread: flat = tid + q * PRODUCERS -> row = flat / 4 over the 384 rows (train rows
-        // first), chunk = flat % 4: four lanes read one row's 128 contiguous bytes, and with the 64-byte
-        // swizzle the 16-byte stores of eight consecutive lanes (two rows) fill 128 contiguous bytes
-        float raw[RING][TASKS][8];
-        auto fetch = [&](int64_t kt, float (&dst)[TASKS][8]) {
-            const int64_t d0 = kt * BK;
-#pragma unroll
-            for (int q = 0; q < TASKS; ++q) {
-                const int flat = tid + q * PRODUCERS;
-                const int row = flat / CHUNKS, ch = flat % CHUNKS;
-                const bool is_a = row < BM;
-                const int64_t gr = is_a ? (n0 + row) : (m0 + (row - BM));
-                const bool row_ok = is_a ? (gr < N) : (gr < M);
-                const float* src = (is_a ? train + gr * ld_train : test + gr * ld_test) + d0 + ch * 8;
-                const int64_t d = d0 + ch * 8;
-                if (row_ok && vec_ok && d + 7 < D) {
-                    const float4 u = __ldg(reinterpret_cast<const float4*>(src));
-                    const float4 w = __ldg(reinterpret_cast<const float4*>(src) + 1);
-                    dst[q][0] = u.x; dst[q][1] = u.y; dst[q][2] = u.z; dst[q][3] = u.w;
-                    dst[q][4] = w.x; dst[q][5] = w.y; dst[q][6] = w.z; dst[q][7] = w.w;
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) dst[q][e] = (row_ok && d + e < D) ? __ldg(src + e) : 0.0f;
-                }
-            }
-        };
-        auto stash = [&](int s, const float (&srcv)[TASKS][8]) {
+        // task q of this thread: flat = tid + q * PRODUCERS -> row = flat / 4 over the 256 staged rows (128
+        // train rows, then this CTA's half of the test rows), chunk = flat % 4 (8 k-values = 32 raw bytes).
+        // Raw tiles carry the 128-byte swizzle (16-byte unit u of row r sits at u ^ (r & 7)), operand tiles
+        // the 64-byte one: both the 16-byte loads and the 16-byte stores of a quarter warp are conflict-free.
+        const unsigned char* raw0 = smem + STAGES * STAGE_BYTES;
+        auto stash = [&](int s, int slot) {
             unsigned char* st = smem + (size_t)s * STAGE_BYTES;
 #pragma unroll
             for (int q = 0; q < TASKS; ++q) {
@@ -116,8 +182,12 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
                 const int row = flat / CHUNKS, ch = flat % CHUNKS;
                 const bool is_a = row < BM;
                 const int r = is_a ? row : row - BM;
+                const unsigned char* rt = raw0 + slot * RAW_BYTES + (is_a ? 0 : RAW_HALF) + r * 128;
+                const float4 u = *reinterpret_cast<const float4*>(rt + (((2 * ch) ^ (r & 7)) << 4));
+                const float4 w = *reinterpret_cast<const float4*>(rt + (((2 * ch + 1) ^ (r & 7)) << 4));
+                const float x[8] = {u.x, u.y, u.z, u.w, w.x, w.y, w.z, w.w};
                 uint4 hi, mid, lo;
-                split8(srcv[q], hi, mid, lo);
+                split8(x, hi, mid, lo);
                 unsigned char* base = is_a ? st : st + 3 * A_SPLIT_BYTES;
                 const int piece = is_a ? A_SPLIT_BYTES : B_SPLIT_BYTES;
                 const uint32_t off = operand_chunk_offset(r, ch);
@@ -126,28 +196,25 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
                 *reinterpret_cast<uint4*>(base + 2 * piece + off) = lo;
             }
         };
-#pragma unroll
-        for (int q = 0; q < PF; ++q)
-            if (q < ktiles) fetch(q, raw[q]);
+        const uint32_t leader_full0 = map_to_cta(full0, 0);
         bool ok = true;
-        for (int64_t kt0 = 0; kt0 < ktiles && ok; kt0 += RING) {
-#pragma unroll
-            for (int ph = 0; ph < RING; ++ph) {
-                const int64_t kt = kt0 + ph;
-                if (kt >= ktiles || !ok) break;
-                const int s = (int)(kt % STAGES);
-                const uint32_t round = (uint32_t)(kt / STAGES);
-                if (kt + PF < ktiles) fetch(kt + PF, raw[(ph + PF) % RING]);
-                if (round > 0) ok = mbar_wait(empty0 + 8 * s, (round - 1) & 1) && !abort_flag;
-                if (!ok) break;
-                stash(s, raw[ph]);
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_arrive(full0 + 8 * s);
+        for (int64_t kt = 0; kt < ktiles; ++kt) {
+            const int s = (int)(kt % STAGES), slot = (int)(kt % RING);
+            const uint32_t round = (uint32_t)(kt / STAGES);
+            ok = mbar_wait(rawfull0 + 8 * slot, (uint32_t)(kt / RING) & 1) && !abort_flag;      // raw tile landed
+            if (ok && round > 0) ok = mbar_wait(empty0 + 8 * s, (round - 1) & 1) && !abort_flag;   // operand stage free
+            if (!ok) break;
+            stash(s, slot);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive_cluster(leader_full0 + 8 * s);
+                mbar_arrive(rawempty0 + 8 * slot);
             }
         }
         if (!ok) abort_flag = 1;
 
-        // ---------------- epilogue: drain the accumulator ----------------
+        // ---------------- epilogue: drain this CTA's accumulators ----------------
         if (ok && ktiles > 0) ok = mbar_wait(accum, 0) && !abort_flag;
         if (!ok) abort_flag = 1;
         ok = __all_sync(0xFFFFFFFFu, ok);   // tensor-memory loads below are warp-collective
@@ -182,14 +249,35 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
                 }
             }
         }
-    } else if (lane == 0) {
-        // ---------------- MMA issuer ----------------
-        const uint32_t idesc = make_idesc(BM, n_mma);
+    } else if (warp == PWARPS + 1) {
+        // ---------------- TMA: raw fp32 tiles into the ring ----------------
+        if (lane == 0) {
+            const uint32_t raw_u32 = smem_base + STAGES * STAGE_BYTES;
+            const int32_t row_a = (int32_t)n0, row_b = (int32_t)(m0 + (int64_t)rank * n_half);
+            int64_t issued = 0;
+            for (int64_t kt = 0; kt < ktiles; ++kt) {
+                const int slot = (int)(kt % RING);
+                if (kt >= RING && !(mbar_wait(rawempty0 + 8 * slot, (uint32_t)(kt / RING - 1) & 1) && !abort_flag)) {
+                    abort_flag = 1;
+                    break;
+                }
+                mbar_expect_tx(rawfull0 + 8 * slot, RAW_BYTES);
+                tma_load_2d(raw_u32 + slot * RAW_BYTES, &map_train, (int32_t)(kt * BK), row_a, rawfull0 + 8 * slot);
+                tma_load_2d(raw_u32 + slot * RAW_BYTES + RAW_HALF, &map_test, (int32_t)(kt * BK), row_b, rawfull0 + 8 * slot);
+                issued = kt + 1;
+            }
+            // no copy of this CTA may still be in flight when it leaves (immediate unless the CTA gave up early)
+            for (int64_t kt = issued > RING ? issued - RING : 0; kt < issued; ++kt)
+                if (!mbar_wait(rawfull0 + 8 * (int)(kt % RING), (uint32_t)(kt / RING) & 1)) abort_flag = 1;
+        }
+    } else if (lane == 0 && rank == 0) {
+        // ---------------- MMA issuer (leader CTA only) ----------------
+        const uint32_t idesc = make_idesc(2 * BM, n_mma);
         bool ok = true;
         for (int64_t kt = 0; kt < ktiles && ok; ++kt) {
             const int s = (int)(kt % STAGES);
             const uint32_t round = (uint32_t)(kt / STAGES);
-            ok = mbar_wait(full0 + 8 * s, round & 1) && !abort_flag;
+            ok = mbar_wait_cluster(full0 + 8 * s, round & 1) && !abort_flag;
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t a0 = smem_base + s * STAGE_BYTES, b0 = a0 + 3 * A_SPLIT_BYTES;
@@ -204,40 +292,82 @@ grass_score_tc_kernel(const float* __restrict__ train, int64_t N, int64_t ld_tra
                     const uint64_t ad = make_smem_desc(a0 + pa[t] * A_SPLIT_BYTES + ks * 32);   // 16 k values on
                     const uint64_t bd = make_smem_desc(b0 + pb[t] * B_SPLIT_BYTES + ks * 32);
                     const uint32_t acc_on = (kt > 0 || ks > 0 || t > 1) ? 1u : 0u;
-                    umma_bf16(t == 0 ? tmem_d : tmem_d + BN, ad, bd, idesc, acc_on);
+                    umma_bf16_pair(t == 0 ? tmem_d : tmem_d + BN, ad, bd, idesc, acc_on);
                 }
             }
-            umma_commit(empty0 + 8 * s);   // stage s may be overwritten once these MMAs have read it
+            umma_commit_pair(empty0 + 8 * s);   // stage s of both CTAs may be overwritten once these MMAs are done
         }
         if (!ok) abort_flag = 1;
-        if (ok && ktiles > 0) umma_commit(accum);   // accumulator complete
+        if (ok && ktiles > 0) umma_commit_pair(accum);   // accumulators of both CTAs complete
     }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    cluster_sync_all();            // nobody leaves while the other CTA may still signal it or read its tiles
     if (warp == PWARPS) {
         __syncwarp();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(TMEM_COLS) : "memory");
     }
 }
 
 }  // namespace tc
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link libcuda)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return (EncodeTiledFn)p;
+    }();
+    return fn;
+}
+
+// rows x D fp32 matrix with row stride ld, read in boxes of 128 rows x 32 k-values (128 bytes, 128-byte swizzle);
+// elements outside the matrix are delivered as zeros
+static bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t D, int64_t ld)
+{
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)ld * sizeof(float)};
+    const cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)tc::BM};
+    const cuuint32_t estride[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), gdim, gstride, box, estride,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// true if the tensor-core path can take these operands (TMA wants 16-byte aligned bases and row strides)
+bool score_tc_supported(const float* train, int64_t ld_train, const float* test, int64_t ld_test, int64_t D)
+{
+    return D > 0 && ((uintptr_t)train % 16 == 0) && ((uintptr_t)test % 16 == 0) && (ld_train % 4 == 0) &&
+           (ld_test % 4 == 0) && encode_tiled_fn() != nullptr;
+}
+
 grass_status launch_score_tc(const float* train, int64_t N, int64_t ld_train, const float* test, int64_t M,
                              int64_t ld_test, int64_t D, float* scores, int64_t ld_s, cudaStream_t st)
 {
-    const int64_t gx = (N + tc::BM - 1) / tc::BM, gy = (M + tc::BN - 1) / tc::BN;
-    if (gx > 0x7FFFFFFFLL || gy > 65535) return GRASS_ERR_UNSUPPORTED;
-    const int vec_ok = ((uintptr_t)train % 16 == 0) && ((uintptr_t)test % 16 == 0) && (ld_train % 4 == 0) &&
-                       (ld_test % 4 == 0);
-    const size_t smem = (size_t)tc::STAGES * tc::STAGE_BYTES + 1024;
+    const int64_t gx = ((N + tc::BM - 1) / tc::BM + 1) / 2 * 2;   // CTA pairs: an even number of row tiles
+    const int64_t gy = (M + tc::BN - 1) / tc::BN;
+    if (gx > 0x7FFFFFFFLL || gy > 65535 || N > 0x7FFFFFFFLL || M > 0x7FFFFFFFLL || D > 0x7FFFFFFFLL)
+        return GRASS_ERR_UNSUPPORTED;
+    CUtensorMap map_train, map_test;
+    if (!make_map(&map_train, train, N, D, ld_train) || !make_map(&map_test, test, M, D, ld_test)) return GRASS_ERR_CUDA;
+    const size_t smem = (size_t)tc::SMEM_BYTES + 1024;
     if (cudaFuncSetAttribute(tc::grass_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
         return GRASS_ERR_CUDA;
     dim3 grid((unsigned)gx, (unsigned)gy);
     const int out_vec_ok = ((uintptr_t)scores % 16 == 0) && (ld_s % 4 == 0);
-    tc::grass_score_tc_kernel<<<grid, tc::THREADS, smem, st>>>(train, N, ld_train, test, M, ld_test, D, scores, ld_s,
-                                                               vec_ok, out_vec_ok);
+    tc::grass_score_tc_kernel<<<grid, tc::THREADS, smem, st>>>(map_train, map_test, N, M, D, scores, ld_s, out_vec_ok);
     return launch_status();
 }
 

@@ -384,7 +384,8 @@ def test_factgrass_grouped_mixed_layers(G, W, oracle_mod):
 
 # ------------------------------------------------------------------ grass_score
 
-@pytest.mark.parametrize("N,M,D", [(300, 70, 257), (128, 128, 64), (1, 1, 1), (513, 256, 4096), (5, 3, 10)])
+@pytest.mark.parametrize("N,M,D", [(300, 70, 257), (128, 128, 64), (1, 1, 1), (513, 256, 4096), (5, 3, 10),
+                                   (300, 70, 260), (200, 24, 96), (130, 300, 64), (1, 1, 4), (257, 8, 36)])
 def test_grass_score_parity(G, W, oracle_mod, N, M, D):
     tr, te = W.score_vectors(N, M, D, 31, device="cuda")
     sc = G.grass_score(tr, te).cpu().numpy()
