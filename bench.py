@@ -450,6 +450,38 @@ def cpu_baseline(cfg_id, W, min_seconds=10.0, max_repeats=20000):
             "kind": "oracle", "sample": what, "seconds": dt}
 
 
+def fig4_microbench(device, G, W, steps=20):
+    """Plain SJLT (identity mask) at p = 131,072 for several input sparsities and output sizes: the shape of
+    the paper's projection benchmark figure (its data are not available; this reports our kernel only).
+    Per case: time per batch of 1,024 samples and the mean relative error of pairwise distances."""
+    p, n, out = 131_072, 1_024, []
+    flush = L2Flush(device)
+    for zero_prob in (0.0, 0.9, 0.99, 0.999):
+        g = W.dense_gradients(n, p, zero_prob, "normal", 1.0, 4242, device=device)
+        sub = g[:128].double()
+        d_true = torch.cdist(sub, sub)
+        iu = torch.triu_indices(128, 128, offset=1, device=device)
+        for k in (512, 4_096, 32_768):
+            res = torch.empty((n, k), dtype=torch.float32, device=device)
+            for _ in range(3):
+                G.grass_compress(g, None, k, 1, 0xF164, out=res)
+            pairs = []
+            for _ in range(steps):
+                flush()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                G.grass_compress(g, None, k, 1, 0xF164, out=res)
+                e1.record()
+                pairs.append((e0, e1))
+            torch.cuda.synchronize()
+            ms = sorted(a.elapsed_time(b) for a, b in pairs)[len(pairs) // 2]
+            d_proj = torch.cdist(res[:128].double(), res[:128].double())
+            rel = ((d_proj - d_true).abs() / d_true)[iu[0], iu[1]].mean().item()
+            out.append({"zero_prob": zero_prob, "k": k, "ms_per_batch": ms, "samples_per_s": n / (ms * 1e-3),
+                        "dense_gbs": n * p * 4 / (ms * 1e-3) / 1e9, "pairwise_distance_rel_err": rel})
+    return {"fig4": {"p": p, "n": n, "s": 1, "l2": "flushed before every call", "cases": out}}
+
+
 def reference_arm(args, W):
     """--impl reference: the CPU oracle, as it stands, timed on the host cores."""
     world, rank, _ = int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), 0
@@ -488,6 +520,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--small", action="store_true", help="reduced case for profiler captures (not a bench value)")
+    ap.add_argument("--fig4", action="store_true",
+                    help="plain SJLT at p = 131,072 over input sparsity and k (not a bench line)")
     ap.add_argument("--fp32-inputs", action="store_true", help="configs 3-5: fp32 A and G instead of bf16")
     ap.add_argument("--precondition", action="store_true",
                     help="config 5: projected FIM of the train vectors, damped solve for the test vectors, then scores")
@@ -509,6 +543,10 @@ def main():
     import paper_2505_18976_b200 as G
     G.lib()
     warmup = args.warmup if args.small else max(args.warmup, 3)
+    if args.fig4:
+        if rank == 0:
+            print(json.dumps(fig4_microbench(device, G, W)))
+        return
 
     job = make_job(args.config, device, G, W, small=args.small, seq_len_aware=args.seq_len_aware,
                    fp32_inputs=args.fp32_inputs, precondition=args.precondition)

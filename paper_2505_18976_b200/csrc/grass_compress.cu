@@ -20,7 +20,22 @@ namespace grass {
 
 constexpr int kThreads = 256;
 
-template <typename T, int S, int U, bool S1>
+// four consecutive elements of a row with one vector load (16 bytes of fp32, 8 bytes of bf16)
+__device__ __forceinline__ void load4(const float* p, float (&v)[4])
+{
+    const float4 t = __ldg(reinterpret_cast<const float4*>(p));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&v)[4])
+{
+    const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
+    v[0] = __uint_as_float(t.x << 16); v[1] = __uint_as_float(t.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(t.y << 16); v[3] = __uint_as_float(t.y & 0xFFFF0000u);
+}
+
+// DENSE: identity mask on vector-aligned rows (plain SJLT, the k' = p case of Section 3.3.1).  Rows are then
+// streamed with vector loads, four consecutive positions per thread, and S > 1 samples share each hash.
+template <typename T, int S, int U, bool S1, bool DENSE>
 __global__ void __launch_bounds__(kThreads)
 grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
                       const uint32_t* __restrict__ idx, int64_t kprime, uint32_t k, uint32_t s,
@@ -44,6 +59,52 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
     for (int si = 0; si < S; ++si) rows[si] = g + (i0 + (si < ns ? si : 0)) * ld;
 
     bool bad = false;
+    if constexpr (DENSE) {
+        constexpr int UD = S >= 8 ? 1 : 8 / S;     // vector loads per sample in flight per thread (8 in all)
+        for (int64_t jb = j0 + (int64_t)tid * 4; jb < j1; jb += (int64_t)kThreads * 4 * UD) {
+            float v[UD][S][4];
+#pragma unroll
+            for (int u = 0; u < UD; ++u) {
+                const int64_t j = jb + (int64_t)u * kThreads * 4;
+#pragma unroll
+                for (int si = 0; si < S; ++si) {
+                    if (si < ns && j + 3 < j1) {
+                        load4(rows[si] + j, v[u][si]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            v[u][si][e] = (si < ns && j + e < j1) ? elem<T>::load(rows[si] + j + e) : 0.0f;
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UD; ++u) {
+                const int64_t j = jb + (int64_t)u * kThreads * 4;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    bool any = false;
+#pragma unroll
+                    for (int si = 0; si < S; ++si) any = any || (v[u][si][e] != 0.0f);
+                    if (!any) continue;     // the cost of the projection follows the non-zeros (Section 3.1)
+                    const uint64_t pos = (uint64_t)(j + e);
+                    const uint32_t draws = S1 ? 1u : s;
+                    for (uint32_t r = 0; r < draws; ++r) {
+                        const uint64_t h = sjlt_hash_counter(seed, S1 ? (pos + 1) : (pos * s + r + 1));
+                        const uint32_t b = sjlt_bucket(h, k);
+#pragma unroll
+                        for (int si = 0; si < S; ++si) {
+                            const float x = v[u][si][e];
+                            if (x != 0.0f) {
+                                const float sx = S1 ? sjlt_signed(h, x) : sjlt_signed(h, x) * scale;
+                                if (use_smem) atomicAdd(&bins[(uint32_t)si * k + b], sx);
+                                else atomicAdd(out + (i0 + si) * ld_out + b, sx);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    } else
     for (int64_t jb = j0 + tid; jb < j1; jb += (int64_t)kThreads * U) {
         uint32_t col[U];
         bool ok[U];
@@ -66,6 +127,12 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             if (!ok[u]) continue;
+            // the hash is only worth computing where some sample has a non-zero entry (Section 3.1: the cost of
+            // the projection follows the number of non-zeros)
+            bool any = false;
+#pragma unroll
+            for (int si = 0; si < S; ++si) any = any || (v[u][si] != 0.0f);
+            if (!any) continue;
             const uint64_t j = (uint64_t)(jb + (int64_t)u * kThreads);
             const uint32_t draws = S1 ? 1u : s;
             for (uint32_t r = 0; r < draws; ++r) {
@@ -139,6 +206,7 @@ grass_mask_kernel(const T* __restrict__ g, int64_t p, int64_t ld, const uint32_t
 }
 
 struct CompressPlan {
+    int dense;      // identity mask on vector-aligned rows: streamed with vector loads
     int S;          // samples per CTA
     int jsplit;     // CTAs that share one sample group (split of the masked positions)
     int use_smem;   // k-bin accumulators fit in shared memory
@@ -151,15 +219,18 @@ static int env_int(const char* name, int dflt)
     return v ? std::atoi(v) : dflt;
 }
 
-static CompressPlan plan_compress(int64_t n, int64_t kprime, uint32_t k, int sm_count)
+static CompressPlan plan_compress(int64_t n, int64_t kprime, uint32_t k, int sm_count, bool dense)
 {
     CompressPlan pl;
+    pl.dense = dense;
     const size_t bin_bytes = (size_t)k * sizeof(float);
     const size_t smem_cap = 200 * 1024;
     pl.use_smem = bin_bytes <= smem_cap;
     // One sample per CTA: the hash is a few dozen integer instructions per position, far below what the
     // gathered loads leave idle, so sharing it between samples buys nothing and costs occupancy.
-    int S = env_int("GRASS_COMPRESS_S", 1);
+    // Dense rows are the exception: every position is read, the hash is the larger cost, and two samples share it
+    // where their bins still leave room for several CTAs per SM (four samples measured slower at k = 4,096).
+    int S = env_int("GRASS_COMPRESS_S", dense && bin_bytes * 2 <= 64 * 1024 ? 2 : 1);
     if (S != 1 && S != 2 && S != 4 && S != 8) S = 1;
     while (S > 1 && pl.use_smem && bin_bytes * S > smem_cap) S >>= 1;
     if (!pl.use_smem) S = 1;
@@ -195,7 +266,8 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
                                     const CompressPlan& pl, uint32_t* dev_status, cudaStream_t st)
 {
     const int64_t groups = (n + S - 1) / S;
-    const int64_t j_per_cta = (kprime + pl.jsplit - 1) / pl.jsplit;
+    int64_t j_per_cta = (kprime + pl.jsplit - 1) / pl.jsplit;
+    if (pl.dense) j_per_cta = (j_per_cta + 3) / 4 * 4;      // vector loads start on multiples of four positions
     // 0: one CTA owns the row, plain stores; 1: global reductions into a zeroed row; 2: cluster reduction
     const int accumulate = pl.cluster ? 2 : ((pl.jsplit > 1 || !pl.use_smem) ? 1 : 0);
     const size_t smem = pl.use_smem ? (size_t)S * sp.k * sizeof(float) : 0;
@@ -224,8 +296,12 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
                                            ld_out, j_per_cta, accumulate, use_smem, dev_status);
         return e == cudaSuccess ? launch_status() : GRASS_ERR_CUDA;
     };
-    if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true>);
-    return launch(grass_compress_kernel<T, S, U, false>);
+    if (pl.dense) {
+        if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true, true>);
+        return launch(grass_compress_kernel<T, S, U, false, true>);
+    }
+    if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true, false>);
+    return launch(grass_compress_kernel<T, S, U, false, false>);
 }
 
 template <typename T>
@@ -236,7 +312,9 @@ static grass_status dispatch_compress(const T* g, int64_t n, int64_t p, int64_t 
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
-    const CompressPlan pl = plan_compress(n, kprime, sp.k, sms);
+    const bool dense = idx == nullptr && env_int("GRASS_COMPRESS_DENSE", 1) != 0 &&
+                       (uintptr_t)g % (4 * sizeof(T)) == 0 && ld % 4 == 0;
+    const CompressPlan pl = plan_compress(n, kprime, sp.k, sms, dense);
     if (!pl.cluster && (pl.jsplit > 1 || !pl.use_smem)) {
         cudaError_t e = cudaMemset2DAsync(out, (size_t)ld_out * sizeof(float), 0, (size_t)sp.k * sizeof(float),
                                           (size_t)n, st);
