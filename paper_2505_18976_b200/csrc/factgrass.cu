@@ -396,14 +396,16 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     // come from L2.  The 128 x 128 variant (1 CTA per SM) is kept for comparison runs.
     const int tile = fg_env_int("FACTGRASS_TILE", 64) == 128 && max_kk > 64 ? 128 : 64;
 
-    const bool grouped = workspace != nullptr;
-    if (!grouped && L != 1) return GRASS_ERR_INVALID_ARG;
+    if (!workspace && L != 1) return GRASS_ERR_INVALID_ARG;
+    if (workspace && (workspace_bytes < (size_t)L * sizeof(LayerDesc) || ((uintptr_t)workspace & 15)))
+        return GRASS_ERR_INVALID_ARG;
+    // a single layer travels as a kernel parameter: no descriptor copy, whoever provided a workspace
+    const bool grouped = workspace != nullptr && L > 1;
     LayerDesc single;
     std::memset(&single, 0, sizeof single);
     LayerDesc* dev_descs = nullptr;
     int max_tiles = 1;
     if (grouped) {
-        if (workspace_bytes < (size_t)L * sizeof(LayerDesc) || ((uintptr_t)workspace & 15)) return GRASS_ERR_INVALID_ARG;
         // descriptors are staged on the host stack / heap and copied on the stream
         LayerDesc stack_buf[256];
         LayerDesc* host = L <= 256 ? stack_buf : (LayerDesc*)std::malloc((size_t)L * sizeof(LayerDesc));
