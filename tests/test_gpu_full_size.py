@@ -163,3 +163,49 @@ def test_config5_full_all_layers_one_launch_and_score(G, W, oracle_mod):
     rowsum = tr.double() @ te.double().sum(0)
     absrow = tr.double().abs() @ te.double().abs().sum(0)
     assert torch.all((sc.double().sum(1) - rowsum).abs() <= 1e-5 * absrow)
+
+
+def test_grass_compress_row_longer_than_2_to_31(G, oracle_mod):
+    """One bf16 row of 3 * 10^9 entries (6 GB): index arithmetic beyond 32 bits.  The oracle works on the
+    gathered entries with the identity mask, which is the same thing by definition (the hash argument is the
+    position in the masked vector)."""
+    p, kp, k, seed = 3_000_000_000, 20_000, 1_024, 41
+    g = torch.zeros((1, p), dtype=torch.bfloat16, device="cuda")
+    rng = np.random.default_rng(3)
+    idx = np.unique(np.concatenate([rng.integers(0, p, kp - 3, dtype=np.int64), [0, 2 ** 31 + 5, p - 1]]))
+    idx = idx[idx != 12345].astype(np.uint32)
+    vals = torch.randn(idx.size, device="cuda").to(torch.bfloat16)
+    g[0, torch.from_numpy(idx.astype(np.int64)).cuda()] = vals
+    g[0, 12345] = 7.0                                   # an entry outside the mask must not be read into the result
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = G.grass_compress(g, G.mask_to_device(idx), k, 1, seed, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    gathered = vals.view(torch.uint16).cpu().numpy().reshape(1, -1)
+    ref, absum = oracle_mod.grass(np.ascontiguousarray(gathered), None, k, 1, seed, dtype="bf16")
+    check_close(out.cpu().numpy(), ref, absum, TOL_BF16, 64, what="row longer than 2^31")
+    mk = G.grass_mask(g, G.mask_to_device(idx)).cpu().numpy()
+    assert np.array_equal(mk[0], vals.float().cpu().numpy())
+
+
+def test_factgrass_operand_larger_than_2_to_31_elements(G, W, oracle_mod):
+    """A of 1 x 36,000 x 65,536 bf16 (2.36 * 10^9 elements): row offsets beyond 32 bits.  The oracle gets the
+    gathered columns with identity masks (the same thing by definition)."""
+    T, d_in, d_out, kin, kout, k, seed = 36_000, 65_536, 96, 64, 40, 777, 5
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(12)
+    A = torch.empty((1, T, d_in), dtype=torch.bfloat16, device="cuda")
+    for t0 in range(0, T, 4_000):
+        A[0, t0:t0 + 4_000] = torch.randn((min(4_000, T - t0), d_in), generator=gen, device="cuda").to(torch.bfloat16)
+    Gt = (torch.randn((1, T, d_out), generator=gen, device="cuda") * 1e-3).to(torch.bfloat16)
+    mi = oracle_mod.random_mask(d_in, kin, 1)
+    mo = oracle_mod.random_mask(d_out, kout, 2)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = G.factgrass_compress(A, Gt, G.mask_to_device(mi), G.mask_to_device(mo), k, 1, seed, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    Am = A[:, :, torch.from_numpy(mi.astype(np.int64)).cuda()].contiguous()
+    Gm = Gt[:, :, torch.from_numpy(mo.astype(np.int64)).cuda()].contiguous()
+    ref, absum = oracle_mod.factgrass(W.bits_of(Am), W.bits_of(Gm), np.arange(kin, dtype=np.uint32),
+                                      np.arange(kout, dtype=np.uint32), k, 1, seed)
+    check_close(out.cpu().numpy(), ref, absum, TOL_BF16, T + 64, eps=EPS_TC, what="operand larger than 2^31 elements")
