@@ -482,6 +482,51 @@ def fig4_microbench(device, G, W, steps=20):
     return {"fig4": {"p": p, "n": n, "s": 1, "l2": "flushed before every call", "cases": out}}
 
 
+def compare_compressors(cfg_id, device, G, W, steps=5):
+    """On-box ordering of the compressors of the paper's Tables 1d / 2 on one configuration's shapes:
+    FactGraSS and factorised Mask (this library) next to LoGra, the Gaussian factorised projection, written here
+    with torch matmuls (cuBLAS) as the paper's own baseline is: a comparison arm, not part of the library."""
+    job = FactJob(W.CONFIGS[cfg_id], device, G, W)
+    cfg = job.cfg
+    kin = kout = int(round(cfg.k ** 0.5))                  # LoGra projects each factor to sqrt(k_l)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(99)
+    proj = {}
+    for lay in cfg.layers:
+        for d, kk in ((lay.d_in, kin), (lay.d_out, kout)):
+            if (d, kk) not in proj:
+                proj[(d, kk)] = torch.randn((d, kk), generator=gen, device=device).to(torch.bfloat16)
+    mask_out = torch.empty((cfg.B, len(cfg.layers) * cfg.kin * cfg.kout), dtype=torch.float32, device=device)
+    mask_layers = [dict(l, out_offset=i * cfg.kin * cfg.kout) for i, l in enumerate(job.layers)]
+    mask_group = G.GroupedLayers(mask_layers)
+    logra_out = torch.empty((cfg.B, len(cfg.layers), kin * kout), dtype=torch.float32, device=device)
+
+    def logra():
+        for i, (l, lay) in enumerate(zip(job.layers, cfg.layers)):
+            a = torch.matmul(l["A"], proj[(lay.d_in, kin)])             # B x T x kin
+            g = torch.matmul(l["G"], proj[(lay.d_out, kout)])           # B x T x kout
+            logra_out[:, i] = torch.bmm(a.transpose(1, 2), g).float().reshape(cfg.B, -1)
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    res = {"FactGraSS (SJLT o Mask, this library)": timed(lambda: G.factgrass_compress_grouped(job.group, job.out, job.ws)),
+           "factorised Mask alone (this library)": timed(lambda: G.factmask_compress_grouped(mask_group, mask_out, job.ws)),
+           "LoGra (Gaussian factorised projection, torch/cuBLAS)": timed(logra)}
+    tokens = cfg.B * cfg.T
+    return {"compare": {"workload": cfg.name, "k_per_layer": cfg.k, "mask": f"{cfg.kin}x{cfg.kout}",
+                        "logra_factors": f"{kin}x{kout}",
+                        "ms_per_batch": res, "tokens_per_s": {n: tokens / (ms * 1e-3) for n, ms in res.items()}}}
+
+
 def reference_arm(args, W):
     """--impl reference: the CPU oracle, as it stands, timed on the host cores."""
     world, rank, _ = int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), 0
@@ -520,6 +565,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--small", action="store_true", help="reduced case for profiler captures (not a bench value)")
+    ap.add_argument("--compare", action="store_true",
+                    help="configs 3-5: FactGraSS / factorised Mask (this library) next to a torch LoGra arm (not a bench line)")
     ap.add_argument("--fig4", action="store_true",
                     help="plain SJLT at p = 131,072 over input sparsity and k (not a bench line)")
     ap.add_argument("--fp32-inputs", action="store_true", help="configs 3-5: fp32 A and G instead of bf16")
@@ -546,6 +593,10 @@ def main():
     if args.fig4:
         if rank == 0:
             print(json.dumps(fig4_microbench(device, G, W)))
+        return
+    if args.compare:
+        if rank == 0:
+            print(json.dumps(compare_compressors(args.config if args.config >= 3 else 5, device, G, W)))
         return
 
     job = make_job(args.config, device, G, W, small=args.small, seq_len_aware=args.seq_len_aware,
