@@ -14,13 +14,13 @@
 //   warp 17    one thread brings the raw fp32 tiles (128 rows x 32 k-values each, train and test) from
 //              global memory into a ring of shared-memory slots with TMA (cp.async.bulk.tensor.2d, 128-byte
 //              swizzle, no multicast); rows and k-values beyond the matrices arrive as zeros;
-//   warps 0-15 producers: read a raw slot, split, and write the bf16 pieces into shared memory in the tensor
+//   warps 0-15 producers, in two groups that take alternate k tiles: read a raw slot, split, and write the bf16 pieces into shared memory in the tensor
 //              core's K-major layout with the 64-byte swizzle; one lane per warp then arrives on the LEADER
 //              CTA's "full" barrier (a remote arrive for the second CTA) and frees the raw slot; afterwards
 //              they drain their own CTA's accumulators;
 //   warp 16    allocates / frees tensor memory in both CTAs; in the leader CTA one elected thread issues
 //              the MMAs and commits, multicast to both CTAs, the stage-free and accumulator-ready barriers.
-// Two 48 KB operand stages and three 32 KB raw slots of 32 k-values each.  Every mbarrier wait is bounded:
+// Three 48 KB operand stages and two 32 KB raw slots of 32 k-values each.  Every mbarrier wait is bounded:
 // if one expires the CTA marks its tile with NaN, still frees its tensor memory, and returns; the cluster
 // barriers are reached by every thread of both CTAs unconditionally.
 // The TMA path needs 16-byte aligned bases and row strides; other inputs take the plain FMA kernel
@@ -36,8 +36,8 @@ namespace tc {
 constexpr int BM = 128;            // train rows per CTA (the pair's MMA M is 256)
 constexpr int BN = 256;            // test rows per CTA pair (MMA N, upper bound); each CTA stages half
 constexpr int BNH = BN / 2;
-constexpr int STAGES = 2;          // bf16 operand stages
-constexpr int RING = 3;            // raw fp32 slots filled by TMA
+constexpr int STAGES = 3;          // bf16 operand stages
+constexpr int RING = 2;            // raw fp32 slots filled by TMA
 constexpr int PRODUCERS = 512;     // threads of the producer warps
 constexpr int PWARPS = PRODUCERS / 32;
 constexpr int THREADS = PRODUCERS + 64;   // + the MMA / tensor-memory warp and the TMA warp
@@ -45,7 +45,15 @@ constexpr int A_SPLIT_BYTES = BM * BK * 2;    // one bf16 piece of the train til
 constexpr int B_SPLIT_BYTES = BNH * BK * 2;   // one bf16 piece of this CTA's half of the test tile: 8 KB
 constexpr int STAGE_BYTES = 3 * (A_SPLIT_BYTES + B_SPLIT_BYTES);   // 48 KB
 constexpr int CHUNKS = BK / 8;     // 16-byte chunks (8 bf16) per row per stage
-constexpr int TASKS = (BM + BNH) * CHUNKS / PRODUCERS;   // (row, chunk) tasks per producer per stage = 2
+constexpr int GROUPS = 2;          // producer warps work in two groups that take alternate k tiles
+constexpr int GROUP_THREADS = PRODUCERS / GROUPS;
+constexpr int GROUP_WARPS = PWARPS / GROUPS;
+constexpr int TASKS = (BM + BNH) * CHUNKS / GROUP_THREADS;   // (row, chunk) tasks per producer per k tile = 4
+// Parity waits are only unambiguous if a waiter never lags a barrier by two phases:
+//  - every k tile that uses a given raw slot belongs to the same group (so a group sees all phases of its slots);
+//  - a group's previous tile has already waited for an MMA at least as late as the one two rounds back on any stage.
+static_assert(RING % GROUPS == 0, "all tiles of a raw slot must belong to one producer group");
+static_assert(GROUPS <= STAGES, "operand-stage phases must not be skipped by a producer group");
 constexpr uint32_t TMEM_COLS = 512;   // two fp32 accumulators of BN columns each
 constexpr int RAW_HALF = BM * BK * 4;            // one raw fp32 tile (128 rows x 32 k-values): 16 KB
 constexpr int RAW_BYTES = 2 * RAW_HALF;          // train tile + this CTA's test tile
@@ -143,13 +151,13 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
     const uint32_t rawfull0 = smem_u32(&bars[2 * STAGES + 1]), rawempty0 = rawfull0 + 8 * RING;
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full0 + 8 * s, 2 * PWARPS);   // one arrival per producer warp of both CTAs (used in the leader)
+            mbar_init(full0 + 8 * s, 2 * GROUP_WARPS);   // one arrival per warp of the stage's group in both CTAs
             mbar_init(empty0 + 8 * s, 1);
         }
         mbar_init(accum, 1);
         for (int r = 0; r < RING; ++r) {
             mbar_init(rawfull0 + 8 * r, 1);        // the TMA thread's expect_tx arrival + the bytes
-            mbar_init(rawempty0 + 8 * r, PWARPS);  // one arrival per producer warp
+            mbar_init(rawempty0 + 8 * r, GROUP_WARPS);   // one arrival per warp of the group that read the slot
         }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -169,25 +177,40 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
 
     if (warp < PWARPS) {
         // ---------------- producers ----------------
-        // task q of this thread: flat = tid + q * PRODUCERS -> row = flat / 4 over the 256 staged rows (128
+        // The split of one k tile is a latency chain (shared-memory loads, the arithmetic, stores, the proxy
+        // fence) about as long as the MMAs of a k tile, so two groups of 8 warps work on alternate k tiles.
+        // task q of a thread: flat = (tid % 256) + q * 256 -> row = flat / 4 over the 256 staged rows (128
         // train rows, then this CTA's half of the test rows), chunk = flat % 4 (8 k-values = 32 raw bytes).
         // Raw tiles carry the 128-byte swizzle (16-byte unit u of row r sits at u ^ (r & 7)), operand tiles
         // the 64-byte one: both the 16-byte loads and the 16-byte stores of a quarter warp are conflict-free.
         const unsigned char* raw0 = smem + STAGES * STAGE_BYTES;
-        auto stash = [&](int s, int slot) {
-            unsigned char* st = smem + (size_t)s * STAGE_BYTES;
+        float x[TASKS][8];
+        // raw slot -> registers (the slot can be refilled as soon as every warp of the group has done this)
+        auto grab = [&](int slot) {
 #pragma unroll
             for (int q = 0; q < TASKS; ++q) {
-                const int flat = tid + q * PRODUCERS;
+                const int flat = (tid % GROUP_THREADS) + q * GROUP_THREADS;
                 const int row = flat / CHUNKS, ch = flat % CHUNKS;
                 const bool is_a = row < BM;
                 const int r = is_a ? row : row - BM;
                 const unsigned char* rt = raw0 + slot * RAW_BYTES + (is_a ? 0 : RAW_HALF) + r * 128;
                 const float4 u = *reinterpret_cast<const float4*>(rt + (((2 * ch) ^ (r & 7)) << 4));
                 const float4 w = *reinterpret_cast<const float4*>(rt + (((2 * ch + 1) ^ (r & 7)) << 4));
-                const float x[8] = {u.x, u.y, u.z, u.w, w.x, w.y, w.z, w.w};
+                x[q][0] = u.x; x[q][1] = u.y; x[q][2] = u.z; x[q][3] = u.w;
+                x[q][4] = w.x; x[q][5] = w.y; x[q][6] = w.z; x[q][7] = w.w;
+            }
+        };
+        // registers -> the three bf16 pieces of operand stage s
+        auto stash = [&](int s) {
+            unsigned char* st = smem + (size_t)s * STAGE_BYTES;
+#pragma unroll
+            for (int q = 0; q < TASKS; ++q) {
+                const int flat = (tid % GROUP_THREADS) + q * GROUP_THREADS;
+                const int row = flat / CHUNKS, ch = flat % CHUNKS;
+                const bool is_a = row < BM;
+                const int r = is_a ? row : row - BM;
                 uint4 hi, mid, lo;
-                split8(x, hi, mid, lo);
+                split8(x[q], hi, mid, lo);
                 unsigned char* base = is_a ? st : st + 3 * A_SPLIT_BYTES;
                 const int piece = is_a ? A_SPLIT_BYTES : B_SPLIT_BYTES;
                 const uint32_t off = operand_chunk_offset(r, ch);
@@ -198,19 +221,20 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
         };
         const uint32_t leader_full0 = map_to_cta(full0, 0);
         bool ok = true;
-        for (int64_t kt = 0; kt < ktiles; ++kt) {
+        for (int64_t kt = warp / GROUP_WARPS; kt < ktiles; kt += GROUPS) {
             const int s = (int)(kt % STAGES), slot = (int)(kt % RING);
             const uint32_t round = (uint32_t)(kt / STAGES);
             ok = mbar_wait(rawfull0 + 8 * slot, (uint32_t)(kt / RING) & 1) && !abort_flag;      // raw tile landed
-            if (ok && round > 0) ok = mbar_wait(empty0 + 8 * s, (round - 1) & 1) && !abort_flag;   // operand stage free
             if (!ok) break;
-            stash(s, slot);
+            grab(slot);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(rawempty0 + 8 * slot);                                     // slot may be refilled
+            if (round > 0) ok = mbar_wait(empty0 + 8 * s, (round - 1) & 1) && !abort_flag;         // operand stage free
+            if (!ok) break;
+            stash(s);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive_cluster(leader_full0 + 8 * s);
-                mbar_arrive(rawempty0 + 8 * slot);
-            }
+            if (lane == 0) mbar_arrive_cluster(leader_full0 + 8 * s);
         }
         if (!ok) abort_flag = 1;
 
