@@ -24,6 +24,7 @@ namespace grass {
 
 constexpr int kFgThreads = 256;
 constexpr int kTokTile = 32;  // tokens per pipeline stage
+constexpr int kFgBufs = 2;    // operand-tile buffers per CTA
 
 struct LayerDesc {
     const void* A;
@@ -75,7 +76,7 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     constexpr int A_TILE = TM * (int)tc::ROW_BYTES;       // one piece of the A operand tile (TM rows x 32 tokens)
     constexpr int G_TILE = TN * (int)tc::ROW_BYTES;
     constexpr int STAGE = NP * (A_TILE + G_TILE);
-    constexpr int NBUF = 2;
+    constexpr int NBUF = kFgBufs;
     constexpr int GA = kFgThreads / TM, GG = kFgThreads / TN;   // 8-token groups covered by one pass
     constexpr int PASS_A = 4 / GA, PASS_G = 4 / GG;             // passes per 32-token stage
     constexpr uint32_t ACC_COLS = F32 ? 2 * TN : TN;            // fp32 accumulator columns in tensor memory
@@ -443,7 +444,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     const size_t bins_bytes = epi == kEpiSjlt ? (size_t)max_k_smem * sizeof(float) : 0;
     const bool f32 = dt == GRASS_F32;
     auto launch = [&](auto kern, size_t stage_bytes) -> grass_status {
-        const size_t smem = 2 * stage_bytes + bins_bytes;
+        const size_t smem = kFgBufs * stage_bytes + bins_bytes;
         // static shared memory counts toward the 48 KB default limit too
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return GRASS_ERR_CUDA;
@@ -550,7 +551,7 @@ grass_status launch_fim(const float* X, int64_t n, int64_t k, int64_t ld, float 
     if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
     auto kern = factgrass_kernel<tile, tile, true, kEpiRaw>;
-    const size_t smem = 2 * 3 * (size_t)tile * tc::ROW_BYTES * 2;
+    const size_t smem = kFgBufs * 3 * (size_t)tile * tc::ROW_BYTES * 2;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return GRASS_ERR_CUDA;
     const int per_sm = 2;   // 97 KB of shared memory and 256 tensor-memory columns per CTA; 196 KB carve-out
