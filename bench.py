@@ -646,8 +646,8 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel per launch, from ncu captures
 # summarised under profiles/ (bytes; None until captured)
-TRAFFIC = {1: 65_797_632 + 326_400, 2: 8 * (425_576_704 + 3_593_984), 3: 124_360_704 + 4_261_888,
-           4: 3 * (1_354_085_000 + 4_346_368), 5: 16 * (1_191_550_000 + 5_442_560)}
+TRAFFIC = {1: 65_799_424 + 336_896, 2: 8 * (425_585_920 + 4_569_856), 3: 124_359_424 + 3_895_296,
+           4: 3 * (1_354_089_000 + 4_009_216), 5: 16 * (1_191_565_000 + 5_072_128)}
 
 if __name__ == "__main__":
     main()
