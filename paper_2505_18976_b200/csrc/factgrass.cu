@@ -1,9 +1,11 @@
 // factgrass_compress: FactGraSS for linear layers (Section 3.3.2) as one fused kernel.
 //
-//   stage 1 (sparsification)  gather A[b,t,mask_in], G[b,t,mask_out] straight from HBM into
-//                             token-major bf16 tiles in shared memory;
+//   stage 1 (sparsification)  gather A[b,t,mask_in], G[b,t,mask_out] straight from HBM; every thread owns
+//                             one masked column and writes 8 consecutive tokens of it as one 16-byte chunk
+//                             of a K-major, 64-byte-swizzled tensor-core operand tile in shared memory;
 //   stage 2 (reconstruction)  C[a,c] += sum_t a'_t[a] * b'_t[c]   (Eq. 2 with selection matrices)
-//                             on tensor cores, bf16 in / fp32 accumulate, tokens = contraction dim;
+//                             with tcgen05.mma, bf16 in / fp32 accumulate in tensor memory, tokens =
+//                             contraction dim; fp32 factors as three exact bf16 pieces and six products;
 //   stage 3 (sparse proj.)    every accumulator entry q = a*kout + c is hashed from the seed and
 //                             added into a k-bin accumulator in shared memory, which is flushed to
 //                             the output row with coalesced reductions.
@@ -393,8 +395,8 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
         if (layers[l].out_offset < 0 || layers[l].out_offset + (int64_t)layers[l].spec.k > ld_out)
             return GRASS_ERR_INVALID_ARG;
     }
-    // 64 x 64 block tiles (3 CTAs per SM); larger blocks are covered by several tiles whose shared rows
-    // come from L2.  The 128 x 128 variant (1 CTA per SM) is kept for comparison runs.
+    // 64 x 64 block tiles; larger blocks are covered by several tiles whose shared rows come from L2.
+    // The 128 x 128 variant serves the projected FIM and comparison runs (FACTGRASS_TILE=128).
     const int tile = fg_env_int("FACTGRASS_TILE", 64) == 128 && max_kk > 64 ? 128 : 64;
 
     if (!workspace && L != 1) return GRASS_ERR_INVALID_ARG;

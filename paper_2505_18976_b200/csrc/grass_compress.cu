@@ -9,6 +9,8 @@
 // split over up to 8 CTAs, those CTAs form a thread-block cluster and add their bins through distributed
 // shared memory, each CTA storing one slice of the row: no zero-fill pass and no global atomics.  Wider
 // splits (few samples, very long masks) fall back to a zero-fill plus global reductions.
+// With the identity mask on vector-aligned rows (plain SJLT) the rows are streamed with 16-byte loads instead
+// of gathers.  grass_mask (Mask alone, Section 3.2) is the gather without the projection.
 #include "grass_common.cuh"
 
 #include <cooperative_groups.h>
