@@ -14,7 +14,8 @@
 //   warp 17    one thread brings the raw fp32 tiles (128 rows x 32 k-values each, train and test) from
 //              global memory into a ring of shared-memory slots with TMA (cp.async.bulk.tensor.2d, 128-byte
 //              swizzle, each CTA loading only for itself); rows and k-values beyond the matrices arrive as zeros;
-//   warps 0-15 producers, in two groups that take alternate k tiles: read a raw slot, split, and write the bf16 pieces into shared memory in the tensor
+//   warps 0-15 producers, in two groups that take alternate k tiles: read a raw slot, split, and write the
+//              bf16 pieces into shared memory in the tensor
 //              core's K-major layout with the 64-byte swizzle; one lane per warp then arrives on the LEADER
 //              CTA's "full" barrier (a remote arrive for the second CTA) and frees the raw slot; afterwards
 //              they drain their own CTA's accumulators;
