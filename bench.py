@@ -507,6 +507,19 @@ def compare_compressors(cfg_id, device, G, W, steps=5):
             g = torch.matmul(l["G"], proj[(lay.d_out, kout)])           # B x T x kout
             logra_out[:, i] = torch.bmm(a.transpose(1, 2), g).float().reshape(cfg.B, -1)
 
+    # factorised SJLT without reconstruction (the paper's SJLT_{k_in (x) k_out} row): every token row of A and G is
+    # projected on its own, then the k_in x k_out block is the token sum of the projected factors; composed of three
+    # calls of this library per layer, the projected factors (a few MB) going through HBM
+    fa = torch.empty((cfg.B * cfg.T, kin), dtype=torch.float32, device=device)
+    fg = torch.empty((cfg.B * cfg.T, kout), dtype=torch.float32, device=device)
+    fs_out = torch.empty((cfg.B, len(cfg.layers), kin * kout), dtype=torch.float32, device=device)
+
+    def fact_sjlt():
+        for i, (l, lay) in enumerate(zip(job.layers, cfg.layers)):
+            G.grass_compress(l["A"].view(cfg.B * cfg.T, lay.d_in), None, kin, 1, 1000 + i, out=fa)
+            G.grass_compress(l["G"].view(cfg.B * cfg.T, lay.d_out), None, kout, 1, 2000 + i, out=fg)
+            G.factmask_compress(fa.view(cfg.B, cfg.T, kin), fg.view(cfg.B, cfg.T, kout), None, None, out=fs_out[:, i])
+
     def timed(fn):
         fn()
         torch.cuda.synchronize()
@@ -520,6 +533,7 @@ def compare_compressors(cfg_id, device, G, W, steps=5):
 
     res = {"FactGraSS (SJLT o Mask, this library)": timed(lambda: G.factgrass_compress_grouped(job.group, job.out, job.ws)),
            "factorised Mask alone (this library)": timed(lambda: G.factmask_compress_grouped(mask_group, mask_out, job.ws)),
+           "factorised SJLT without reconstruction (this library, three calls per layer)": timed(fact_sjlt),
            "LoGra (Gaussian factorised projection, torch/cuBLAS)": timed(logra)}
     tokens = cfg.B * cfg.T
     return {"compare": {"workload": cfg.name, "k_per_layer": cfg.k, "mask": f"{cfg.kin}x{cfg.kout}",

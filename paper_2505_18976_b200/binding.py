@@ -318,11 +318,13 @@ def factmask_compress(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, m
     assert A.is_contiguous() and G.is_contiguous() and A.dim() == 3 and G.dim() == 3 and A.dtype == G.dtype
     B, T, d_in = A.shape
     d_out = G.shape[2]
-    kp = mask_in.numel() * mask_out.numel()
+    kin = d_in if mask_in is None else mask_in.numel()          # None = identity mask
+    kout = d_out if mask_out is None else mask_out.numel()
+    kp = kin * kout
     if out is None:
         out = torch.empty((B, kp), dtype=torch.float32, device=A.device)
-    _check(lib().factmask_compress(_ptr(A), _ptr(G), _dt(A), B, T, d_in, d_out, _ptr(mask_in), mask_in.numel(),
-                                   _ptr(mask_out), mask_out.numel(), _ptr(out),
+    _check(lib().factmask_compress(_ptr(A), _ptr(G), _dt(A), B, T, d_in, d_out, _ptr(mask_in), kin,
+                                   _ptr(mask_out), kout, _ptr(out),
                                    out.stride(0) if B > 1 else max(out.shape[1], kp), _ptr(dev_status), _stream()),
            "factmask_compress")
     return out
