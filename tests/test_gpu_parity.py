@@ -393,6 +393,23 @@ def test_grass_score_parity(G, W, oracle_mod, N, M, D):
     check_close(sc, ref, absum, TOL_F32, D + 8, what=f"score {N}x{M}x{D}")
 
 
+def test_grass_score_many_aligned_shapes(G, W, oracle_mod):
+    """Seeded sweep over shapes that take the tensor-core path (row strides a multiple of four floats): row
+    counts around the 128 / 256 tile edges, several column tiles, k extents that end inside a 32-wide k tile,
+    and operands that are column slices of wider matrices."""
+    rng = np.random.default_rng(77)
+    shapes = [(127, 255, 28), (129, 257, 36), (255, 1, 4), (256, 256, 32), (257, 513, 100), (384, 16, 2052),
+              (1, 300, 64), (640, 40, 8)]
+    shapes += [(int(rng.integers(1, 700)), int(rng.integers(1, 600)), 4 * int(rng.integers(1, 300))) for _ in range(6)]
+    for (N, M, D) in shapes:
+        pad = 4 * int(rng.integers(0, 3))
+        trw, tew = W.score_vectors(N, M, D + pad, 900 + N, device="cuda")
+        tr, te = trw[:, :D], tew[:, :D]
+        sc = G.grass_score(tr, te).cpu().numpy()
+        ref, absum = oracle_mod.score(np.ascontiguousarray(tr.cpu().numpy()), np.ascontiguousarray(te.cpu().numpy()))
+        check_close(sc, ref, absum, TOL_F32, D + 8, what=f"score {N}x{M}x{D} ld={D + pad}")
+
+
 def test_grass_score_strided_and_compressed_inputs(G, W, oracle_mod):
     """Scores of actual compressed gradients; train rows taken from a wider matrix."""
     g = W.dense_gradients(40, 30_000, 0.7, "normal", 1.0, 9, device="cuda")
