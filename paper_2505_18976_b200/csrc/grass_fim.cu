@@ -33,86 +33,84 @@ __global__ void add_damping_kernel(float* __restrict__ F, int64_t k, int64_t ld,
 // triangle of F is not used by anything else, and with the inverse at hand every triangular solve against
 // this block becomes a small matrix product.  A pivot that is not positive sets GRASS_DEV_NOT_PD and is
 // replaced by 1 so that nothing divides by zero.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(NB)
 potrf_diag_kernel(float* __restrict__ F, int64_t ld, int64_t j0, int jb, uint32_t* dev_status)
 {
-    __shared__ float a[NB][NB + 1];
-    __shared__ float inv[NB][NB + 1];
-    const int tid = threadIdx.x;
+    __shared__ float a[NB][NB + 1];                    // as the block is stored: the factor, and the transposed
+                                                       // inverse above the diagonal
+    __shared__ __align__(16) float lrel[NB][NB];       // lrel[c][m] = L[c+1+m][c], zero beyond the last row
+    __shared__ __align__(16) float colc[2][NB];
+    __shared__ float rdiag[NB];
+    const int j = threadIdx.x;
     float* blk = F + j0 * ld + j0;
-    // rows and columns beyond jb are padded with the identity, so the loops below have fixed bounds
-    {
-        float v[NB * NB / 256];
+    float col[NB];                                     // col[i] = A[i][j]; the loads are all in flight together
 #pragma unroll
-        for (int u = 0; u < NB * NB / 256; ++u) {
-            const int e = tid + u * 256, r = e / NB, c = e % NB;
-            v[u] = (r < jb && c <= r) ? blk[(int64_t)r * ld + c] : ((r == c && r >= jb) ? 1.0f : 0.0f);
-        }
-#pragma unroll
-        for (int u = 0; u < NB * NB / 256; ++u) {
-            const int e = tid + u * 256;
-            a[e / NB][e % NB] = v[u];
-            inv[e / NB][e % NB] = 0.0f;
-        }
-    }
-    // thread (i, jq) owns row i, columns jq, jq + 4, ..., jq + 60
-    const int i = tid >> 2, jq = tid & 3;
+    for (int i = 0; i < NB; ++i)
+        col[i] = (i < jb && j <= i) ? blk[(int64_t)i * ld + j] : ((i == j && i >= jb) ? 1.0f : 0.0f);
+    // Unscaled right-looking elimination: the owner of column c publishes it as it stands, every later column
+    // subtracts A[i][c] A[j][c] / pivot.  Entries above a column's diagonal take part in the arithmetic but are
+    // never read as results, so the update needs no row predicate; columns are scaled by 1/sqrt(pivot) at the end.
+    bool not_pd = false;
+    float pivot = 1.0f;
 #pragma unroll 1
     for (int c = 0; c < NB; ++c) {
-        __syncthreads();
-        float d = a[c][c];
-        if (!(d > 0.0f)) {
-            if (tid == 0 && dev_status) atomicOr(dev_status, GRASS_DEV_NOT_PD);
-            d = 1.0f;
+        float* cc = colc[c & 1];
+        if (j == c) {
+#pragma unroll
+            for (int i4 = 0; i4 < NB; i4 += 4)
+                *reinterpret_cast<float4*>(&cc[i4]) = make_float4(col[i4], col[i4 + 1], col[i4 + 2], col[i4 + 3]);
         }
-        const float sd = sqrtf(d);
-        __syncthreads();
-        if (jq == 0 && i >= c) a[i][c] = (i == c) ? sd : a[i][c] / sd;
-        __syncthreads();
-        if (i > c) {
-            const float lic = a[i][c];
-            float t[NB / 4], l[NB / 4];
+        __syncthreads();                               // colc is double-buffered: one barrier per column
+        float d = cc[c];
+        if (!(d > 0.0f)) { not_pd = true; d = 1.0f; }
+        if (j == c) pivot = d;
+        if (j > c) {
+            const float w = -cc[j] * __frcp_rn(d);
 #pragma unroll
-            for (int m = 0; m < NB / 4; ++m) {           // all loads first: they are independent
-                t[m] = a[i][jq + 4 * m];
-                l[m] = a[jq + 4 * m][c];
-            }
-#pragma unroll
-            for (int m = 0; m < NB / 4; ++m) {
-                const int j = jq + 4 * m;
-                if (j > c && j <= i) a[i][j] = fmaf(-lic, l[m], t[m]);
+            for (int i4 = 0; i4 < NB; i4 += 4) {
+                const float4 l4 = *reinterpret_cast<const float4*>(&cc[i4]);
+                col[i4 + 0] = fmaf(l4.x, w, col[i4 + 0]);
+                col[i4 + 1] = fmaf(l4.y, w, col[i4 + 1]);
+                col[i4 + 2] = fmaf(l4.z, w, col[i4 + 2]);
+                col[i4 + 3] = fmaf(l4.w, w, col[i4 + 3]);
             }
         }
     }
-    __syncthreads();
-    // inverse of the factor by forward substitution: a quad of lanes per column, each lane summing every
-    // fourth term; all lanes run the same number of steps because the shuffles are warp-wide
+    if (not_pd && j == 0 && dev_status) atomicOr(dev_status, GRASS_DEV_NOT_PD);
     {
-        const int col = tid >> 2, part = tid & 3;
+        const float sd = sqrtf(pivot), rs = 1.0f / sd;
+        rdiag[j] = rs;
+#pragma unroll
+        for (int i = 0; i < NB; ++i) if (i >= j) a[i][j] = (i > j) ? col[i] * rs : sd;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int m = 0; m < NB; ++m) lrel[j][m] = (j + 1 + m < NB) ? a[j + 1 + m][j] : 0.0f;
+    __syncthreads();
+    // Inverse of the factor, thread j on column j, by column-oriented forward substitution.  t[m] holds the
+    // running right-hand side of row c+1+m: the window slides down one row per step inside the FMAs, so every
+    // register index is a compile-time constant while c stays a run-time loop.
+    float t[NB];
+#pragma unroll
+    for (int i = 0; i < NB; ++i) t[i] = (i == j) ? 1.0f : 0.0f;
 #pragma unroll 1
-        for (int r = 0; r < NB; ++r) {
-            float fa[NB / 4], fx[NB / 4];
+    for (int c = 0; c < NB; ++c) {
+        const float x = t[0] * rdiag[c];
+        if (c > j) a[j][c] = x;
+        const float nx = -x;
 #pragma unroll
-            for (int m = 0; m < NB / 4; ++m) {
-                fa[m] = a[r][part + 4 * m];
-                fx[m] = inv[part + 4 * m][col];          // zero above the diagonal and where not yet computed
-            }
-            float v = 0.0f;
-#pragma unroll
-            for (int m = 0; m < NB / 4; ++m)
-                if (part + 4 * m < r) v = fmaf(-fa[m], fx[m], v);
-            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-            if (part == 0 && r >= col) inv[r][col] = ((r == col ? 1.0f : 0.0f) + v) / a[r][r];
-            __syncwarp();
+        for (int m4 = 0; m4 < NB; m4 += 4) {
+            const float4 l4 = *reinterpret_cast<const float4*>(&lrel[c][m4]);
+            t[m4 + 0] = fmaf(l4.x, nx, t[m4 + 1]);
+            t[m4 + 1] = fmaf(l4.y, nx, t[m4 + 2]);
+            t[m4 + 2] = fmaf(l4.z, nx, t[m4 + 3]);
+            t[m4 + 3] = (m4 + 4 < NB) ? fmaf(l4.w, nx, t[(m4 + 4) & (NB - 1)]) : 0.0f;
         }
     }
     __syncthreads();
-#pragma unroll
-    for (int u = 0; u < NB * NB / 256; ++u) {
-        const int e = tid + u * 256, r = e / NB, c = e % NB;
-        if (r < jb && c < jb) blk[(int64_t)r * ld + c] = (c <= r) ? a[r][c] : inv[c][r];
-    }
+#pragma unroll 8
+    for (int r = 0; r < NB; ++r)
+        if (r < jb && j < jb) blk[(int64_t)r * ld + j] = a[r][j];
 }
 
 // Rows of C (rows x jb, at the block's column offset) solved against the diagonal block through its stored
@@ -258,7 +256,7 @@ extern "C" grass_status grass_fim_factor(float* F, int64_t k, int64_t ld_f, floa
     if (lambda != 0.0f) add_damping_kernel<<<(unsigned)((k + 255) / 256), 256, 0, st>>>(F, k, ld_f, lambda);
     for (int64_t j0 = 0; j0 < k; j0 += NB) {
         const int jb = (int)((k - j0) < NB ? (k - j0) : NB);
-        potrf_diag_kernel<<<1, 256, 0, st>>>(F, ld_f, j0, jb, dev_status);
+        potrf_diag_kernel<<<1, NB, 0, st>>>(F, ld_f, j0, jb, dev_status);
         const int64_t rest = k - j0 - jb;
         if (rest > 0) {
             float* panel = F + (j0 + jb) * ld_f + j0;            // rows below the diagonal block, its columns
