@@ -61,6 +61,10 @@ class ClockSampler:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
                  "-lms", "25"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            # the tool needs a moment to start: wait for its first line so that a short timed region is covered
+            t_end = time.time() + 3.0
+            while time.time() < t_end and os.path.getsize(self.path) == 0 and self.proc.poll() is None:
+                time.sleep(0.01)
         except Exception:
             self.proc = None
 
@@ -482,6 +486,36 @@ def fig4_microbench(device, G, W, steps=20):
     return {"fig4": {"p": p, "n": n, "s": 1, "l2": "flushed before every call", "cases": out}}
 
 
+def score_full_concatenation(device, G, W, steps=5):
+    """grass_score over config 5's whole compressed vector: train 16,384 x 917,504 fp32 (60 GB, far beyond L2),
+    test 256 x 917,504.  Reported beside the per-layer-block shape the default step times; not a bench line."""
+    c = W.CONFIG5
+    N, M, D = c.score_n_train, c.score_n_test, c.out_dim
+    gen = torch.Generator(device=device)
+    gen.manual_seed(c.data_seed + 9)
+    tr = torch.empty((N, D), dtype=torch.float32, device=device)
+    for i in range(0, N, 1_024):
+        tr[i:i + 1_024].normal_(generator=gen)
+    te = torch.randn((M, D), generator=gen, device=device)
+    out = torch.empty((N, M), dtype=torch.float32, device=device)
+    for _ in range(2):
+        G.grass_score(tr, te, out=out)
+    pairs = []
+    for _ in range(steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        G.grass_score(tr, te, out=out)
+        e1.record()
+        pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    ms = sorted(a.elapsed_time(b) for a, b in pairs)[len(pairs) // 2]
+    peaks, src = load_peaks()
+    tf = 2.0 * N * M * D / (ms * 1e-3) / 1e12
+    return {"score_full": {"N": N, "M": M, "D": D, "ms": ms, "fp32_equivalent_tflops": tf,
+                           "bf16_product_tflops": 6 * tf, "frac_of_bf16_peak": 6 * tf / peaks["bf16_tflops"],
+                           "peak_source": src, "train_gbs": N * D * 4 / (ms * 1e-3) / 1e9}}
+
+
 def compare_compressors(cfg_id, device, G, W, steps=5):
     """On-box ordering of the compressors of the paper's Tables 1d / 2 on one configuration's shapes:
     FactGraSS and factorised Mask (this library) next to LoGra, the Gaussian factorised projection, written here
@@ -583,6 +617,8 @@ def main():
                     help="configs 3-5: FactGraSS / factorised Mask (this library) next to a torch LoGra arm (not a bench line)")
     ap.add_argument("--fig4", action="store_true",
                     help="plain SJLT at p = 131,072 over input sparsity and k (not a bench line)")
+    ap.add_argument("--score-full", action="store_true",
+                    help="grass_score over config 5's full concatenation, D = 917,504 (60 GB; not a bench line)")
     ap.add_argument("--fp32-inputs", action="store_true", help="configs 3-5: fp32 A and G instead of bf16")
     ap.add_argument("--precondition", action="store_true",
                     help="config 5: projected FIM of the train vectors, damped solve for the test vectors, then scores")
@@ -607,6 +643,10 @@ def main():
     if args.fig4:
         if rank == 0:
             print(json.dumps(fig4_microbench(device, G, W)))
+        return
+    if args.score_full:
+        if rank == 0:
+            print(json.dumps(score_full_concatenation(device, G, W)))
         return
     if args.compare:
         if rank == 0:

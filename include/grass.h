@@ -199,7 +199,10 @@ grass_status factgrass_compress_grouped_static(const factgrass_layer* layers /*h
 /*
  * Attribute-stage scores (Section 2.1): scores[i*ld_s + m] = <train[i, :], test[m, :]>.
  *   train N x D, test M x D, fp32 row-major with strides ld_train, ld_test >= D.
- *   scores N x M fp32 (train-major), row stride ld_s >= M.  Overwritten.  fp32 accumulation.
+ *   scores N x M fp32 (train-major), row stride ld_s >= M.  Overwritten (columns beyond M are left alone).
+ *   fp32-accurate products and fp32 accumulation; contractions longer than 16,384 are summed in runs of
+ *   8,192 so that the relative accuracy does not degrade with D.  Whenever the contraction is split (long D,
+ *   or few output tiles) the partial sums meet in the output, which the call first zeroes on the stream.
  * These are raw inner products of compressed gradients; preconditioning is the caller's.
  */
 grass_status grass_score(const float* train, int64_t N, int64_t ld_train, const float* test, int64_t M,

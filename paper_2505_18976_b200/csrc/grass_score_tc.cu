@@ -24,9 +24,14 @@
 // Three 48 KB operand stages and two 32 KB raw slots of 32 k-values each.  Every mbarrier wait is bounded:
 // if one expires the CTA marks its tile with NaN, still frees its tensor memory, and returns; the cluster
 // barriers are reached by every thread of both CTAs unconditionally.
+// Long contractions, and outputs with too few tiles to fill the machine, are split over blockIdx.z: every split
+// adds its partial products into the zeroed output (see launch_score_tc).
 // The TMA path needs 16-byte aligned bases and row strides; other inputs take the plain FMA kernel
 // (grass_score.cu).
 #include <cuda.h>
+
+#include <algorithm>
+#include <cstdlib>
 
 #include "grass_common.cuh"
 #include "tcgen05_util.cuh"
@@ -132,7 +137,8 @@ __device__ __forceinline__ void cluster_sync_all()
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __grid_constant__ CUtensorMap map_test,
-                      int64_t N, int64_t M, int64_t D, float* __restrict__ scores, int64_t ld_s, int out_vec_ok)
+                      int64_t N, int64_t M, int64_t D, int64_t kt_split, float* __restrict__ scores, int64_t ld_s,
+                      int out_vec_ok)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ __align__(8) unsigned long long bars[2 * STAGES + 1 + 2 * RING];
@@ -146,7 +152,12 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
     const int64_t m_rows = (M - m0) < BN ? (M - m0) : BN;          // test rows of the pair's tile
     const uint32_t n_mma = (uint32_t)((m_rows + 15) / 16 * 16);    // MMA N (a multiple of 16 for M = 256)
     const int n_half = (int)(n_mma / 2);                           // test rows staged by each CTA
-    const int64_t ktiles = (D + BK - 1) / BK;
+    // blockIdx.z takes k tiles [kt0, kt0 + ktiles); with more than one split the tiles add their partial
+    // products into the (zeroed) output
+    const int64_t kt0 = (int64_t)blockIdx.z * kt_split;
+    const int64_t kt_left = (D + BK - 1) / BK - kt0;
+    const int64_t ktiles = kt_left < kt_split ? (kt_left > 0 ? kt_left : 0) : kt_split;
+    const bool add_out = gridDim.z > 1;
 
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]), accum = smem_u32(&bars[2 * STAGES]);
     const uint32_t rawfull0 = smem_u32(&bars[2 * STAGES + 1]), rawempty0 = rawfull0 + 8 * RING;
@@ -263,7 +274,21 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
             }
             if (row < N) {
                 float* dst = scores + row * ld_s + m0 + c0;
-                if (out_vec_ok && (int64_t)(c0 + 32) <= m_rows) {
+                const bool vec = out_vec_ok && (int64_t)(c0 + 32) <= m_rows;
+                if (add_out) {
+                    if (vec) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + e),
+                                         "f"(__uint_as_float(v[e])), "f"(__uint_as_float(v[e + 1])),
+                                         "f"(__uint_as_float(v[e + 2])), "f"(__uint_as_float(v[e + 3]))
+                                         : "memory");
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if ((int64_t)(c0 + e) < m_rows) atomicAdd(dst + e, __uint_as_float(v[e]));
+                    }
+                } else if (vec) {
 #pragma unroll
                     for (int e = 0; e < 32; e += 4)
                         *reinterpret_cast<uint4*>(dst + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
@@ -287,8 +312,8 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
                     break;
                 }
                 mbar_expect_tx(rawfull0 + 8 * slot, RAW_BYTES);
-                tma_load_2d(raw_u32 + slot * RAW_BYTES, &map_train, (int32_t)(kt * BK), row_a, rawfull0 + 8 * slot);
-                tma_load_2d(raw_u32 + slot * RAW_BYTES + RAW_HALF, &map_test, (int32_t)(kt * BK), row_b, rawfull0 + 8 * slot);
+                tma_load_2d(raw_u32 + slot * RAW_BYTES, &map_train, (int32_t)((kt0 + kt) * BK), row_a, rawfull0 + 8 * slot);
+                tma_load_2d(raw_u32 + slot * RAW_BYTES + RAW_HALF, &map_test, (int32_t)((kt0 + kt) * BK), row_b, rawfull0 + 8 * slot);
                 issued = kt + 1;
             }
             // no copy of this CTA may still be in flight when it leaves (immediate unless the CTA gave up early)
@@ -390,9 +415,29 @@ grass_status launch_score_tc(const float* train, int64_t N, int64_t ld_train, co
     if (cudaFuncSetAttribute(tc::grass_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
         return GRASS_ERR_CUDA;
-    dim3 grid((unsigned)gx, (unsigned)gy);
+    // Split of the contraction over blockIdx.z, for two reasons.  Accuracy: the tensor core truncates the fp32
+    // accumulator after every MMA, a bias that grows with the number of accumulations, so one accumulator
+    // never runs over more than 8,192 k-values once D exceeds 16,384 (the partial sums are then added in
+    // round-to-nearest fp32).  Occupancy: with fewer tile pairs than SM pairs, k is split until the machine
+    // is about full, in pieces of at least 256 k-values.
+    const int64_t ktiles = (D + tc::BK - 1) / tc::BK;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    const int64_t pairs = gx / 2 * gy;
+    int64_t splits = D > 16384 ? (D + 8191) / 8192 : 1;
+    if (pairs > 0 && pairs * 2 <= sms / 2) splits = std::max<int64_t>(splits, std::min<int64_t>(sms / 2 / pairs, D / 256));
+    if (const char* e = std::getenv("GRASS_SCORE_SPLITS")) splits = std::atoll(e);
+    splits = std::max<int64_t>(1, std::min<int64_t>(splits, std::min<int64_t>(ktiles, 65535)));
+    const int64_t kt_split = (ktiles + splits - 1) / splits;
+    splits = (ktiles + kt_split - 1) / kt_split;
+    if (splits > 1 &&
+        cudaMemset2DAsync(scores, (size_t)ld_s * sizeof(float), 0, (size_t)M * sizeof(float), (size_t)N, st) != cudaSuccess)
+        return GRASS_ERR_CUDA;
+    dim3 grid((unsigned)gx, (unsigned)gy, (unsigned)splits);
     const int out_vec_ok = ((uintptr_t)scores % 16 == 0) && (ld_s % 4 == 0);
-    tc::grass_score_tc_kernel<<<grid, tc::THREADS, smem, st>>>(map_train, map_test, N, M, D, scores, ld_s, out_vec_ok);
+    tc::grass_score_tc_kernel<<<grid, tc::THREADS, smem, st>>>(map_train, map_test, N, M, D, kt_split, scores, ld_s,
+                                                               out_vec_ok);
     return launch_status();
 }
 

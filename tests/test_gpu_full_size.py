@@ -209,3 +209,31 @@ def test_factgrass_operand_larger_than_2_to_31_elements(G, W, oracle_mod):
     ref, absum = oracle_mod.factgrass(W.bits_of(Am), W.bits_of(Gm), np.arange(kin, dtype=np.uint32),
                                       np.arange(kout, dtype=np.uint32), k, 1, seed)
     check_close(out.cpu().numpy(), ref, absum, TOL_BF16, T + 64, eps=EPS_TC, what="operand larger than 2^31 elements")
+
+
+def test_config5_score_over_the_full_concatenation(G, oracle_mod):
+    """Scores over all 224 layers at once: train 16,384 x 917,504 fp32 (60 GB), test 256 x 917,504.  The oracle
+    recomputes sampled train rows; every row is checked against the Cauchy-Schwarz bound and the row-sum identity."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 100 * 2 ** 30:
+        pytest.skip("needs about 95 GB of free device memory")
+    N, M, D = 16_384, 256, 224 * 4_096
+    g = torch.Generator(device="cuda")
+    g.manual_seed(2_005)
+    tr = torch.empty((N, D), dtype=torch.float32, device="cuda")
+    for i in range(0, N, 1_024):
+        tr[i:i + 1_024].normal_(generator=g)
+    te = torch.randn((M, D), generator=g, device="cuda")
+    sc = G.grass_score(tr, te)
+    torch.cuda.synchronize()
+    assert torch.isfinite(sc).all()
+    rows = [0, 127, 128, 255, 256, 8_191, 16_383] + [int(r) for r in np.random.default_rng(8).integers(0, N, 9)]
+    ref, absum = oracle_mod.score(tr[rows].cpu().numpy(), te.cpu().numpy())
+    check_close(sc[rows].cpu().numpy(), ref, absum, TOL_F32, 8_192 + 8 + 112, what="score over D = 917,504, sampled rows")
+    te_sum, te_abs, te_norm = te.double().sum(0), te.double().abs().sum(0), te.double().norm(dim=1)
+    for i in range(0, N, 2_048):
+        blk = tr[i:i + 2_048].double()
+        s = sc[i:i + 2_048].double()
+        assert torch.all(s.abs() <= blk.norm(dim=1)[:, None] * te_norm[None, :] * (1 + 1e-6))
+        assert torch.all((s.sum(1) - blk @ te_sum).abs() <= 1e-5 * (blk.abs() @ te_abs))
+        del blk

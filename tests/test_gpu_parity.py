@@ -421,3 +421,41 @@ def test_grass_score_strided_and_compressed_inputs(G, W, oracle_mod):
     sc = G.grass_score(tr, te).cpu().numpy()
     ref, absum = oracle_mod.score(np.ascontiguousarray(tr.cpu().numpy()), np.ascontiguousarray(te.cpu().numpy()))
     check_close(sc, ref, absum, TOL_F32, 520, what="score of compressed")
+
+
+def test_grass_score_split_contraction(G, W, oracle_mod, monkeypatch):
+    """The contraction split over several CTAs per output tile (partial products added into the zeroed output):
+    forced through the environment switch, with a ragged last split, vector and scalar reductions (output row
+    stride a multiple of four floats or not), stale data in the output buffer; then the two automatic cases,
+    a long contraction (D > 16,384) and a small output that would leave most SMs idle."""
+    for splits, (N, M, D), ld_s in [(3, (300, 70, 260), 70), (5, (129, 257, 1000), 260), (2, (256, 256, 64), 256),
+                                    (64, (40, 300, 128), 301), (7, (513, 24, 4096), 24)]:
+        monkeypatch.setenv("GRASS_SCORE_SPLITS", str(splits))
+        tr, te = W.score_vectors(N, M, D, 55 + splits, device="cuda")
+        buf = torch.full((N, ld_s), 123.0, device="cuda")
+        sc = G.grass_score(tr, te, out=buf[:, :M])
+        ref, absum = oracle_mod.score(tr.cpu().numpy(), te.cpu().numpy())
+        check_close(sc.cpu().numpy(), ref, absum, TOL_F32, D + 8 + splits, what=f"score {N}x{M}x{D}, {splits} splits")
+        if ld_s > M:
+            assert torch.all(buf[:, M:] == 123.0), "columns beyond M must not be touched"
+    monkeypatch.delenv("GRASS_SCORE_SPLITS")
+    for (N, M, D) in [(200, 100, 20_000), (64, 32, 8_192), (300, 520, 3_000)]:
+        tr, te = W.score_vectors(N, M, D, 77, device="cuda")
+        sc = G.grass_score(tr, te, out=torch.full((N, M), -5.0, device="cuda"))
+        ref, absum = oracle_mod.score(tr.cpu().numpy(), te.cpu().numpy())
+        check_close(sc.cpu().numpy(), ref, absum, TOL_F32, D + 64, what=f"score {N}x{M}x{D}, automatic split")
+
+
+def test_grass_score_long_contraction_keeps_relative_accuracy(G, oracle_mod):
+    """Positive operands, D = 262,144: nothing cancels, so every score must be right to 1e-4 relative.  The
+    tensor core truncates its fp32 accumulator after every MMA; a single accumulator over 16,384 MMAs would be
+    biased by several 1e-4, which is why long contractions are split into runs of 8,192 k-values."""
+    N, M, D = 256, 64, 262_144
+    g = torch.Generator(device="cuda")
+    g.manual_seed(12)
+    tr = torch.rand((N, D), generator=g, device="cuda") + 0.5
+    te = torch.rand((M, D), generator=g, device="cuda") + 0.5
+    sc = G.grass_score(tr, te).cpu().numpy().astype(np.float64)
+    ref, _ = oracle_mod.score(tr.cpu().numpy(), te.cpu().numpy())
+    rel = np.abs(sc - ref) / np.abs(ref)
+    assert rel.max() <= 1e-4, rel.max()
