@@ -488,6 +488,9 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
         const int min_chunk = 64;
         int64_t want = base_items < slots ? slots / base_items : (8 * slots + base_items - 1) / base_items;
         int64_t max_chunks = (T + min_chunk - 1) / min_chunk;
+        // the tensor core truncates its fp32 accumulator after every MMA: no accumulator runs over more than
+        // 8,192 tokens, so that this bias stays near 1e-5 of the result however long the sequence is
+        want = std::max<int64_t>(want, ((int64_t)T + 8191) / 8192);
         if (want > max_chunks) want = max_chunks;
         if (want < 1) want = 1;
         int chunk_len = (int)((T + want - 1) / want);
@@ -563,6 +566,7 @@ grass_status launch_fim(const float* X, int64_t n, int64_t k, int64_t ld, float 
     const int64_t tiles = (int64_t)d.tiles_m * (d.tiles_m + 1) / 2;
     int64_t want = (4 * (int64_t)sms * per_sm + tiles - 1) / tiles;
     const int64_t max_chunks = (n + 255) / 256;
+    want = std::max<int64_t>(want, (n + 8191) / 8192);   // bounded accumulation runs, as for the token chunks
     if (want > max_chunks) want = max_chunks;
     if (want < 1) want = 1;
     int64_t chunk_len = (n + want - 1) / want;

@@ -237,3 +237,39 @@ def test_config5_score_over_the_full_concatenation(G, oracle_mod):
         assert torch.all(s.abs() <= blk.norm(dim=1)[:, None] * te_norm[None, :] * (1 + 1e-6))
         assert torch.all((s.sum(1) - blk @ te_sum).abs() <= 1e-5 * (blk.abs() @ te_abs))
         del blk
+
+
+def test_long_accumulations_keep_relative_accuracy(G, W, oracle_mod):
+    """Positive data, so nothing cancels and every output must be right to 1e-4 relative: the projected FIM of
+    400,000 samples at k = 2,048 (enough tiles that each would otherwise sum a third of the samples in one
+    accumulator), and FactGraSS over 32,768 tokens for 1,024 (layer, sample) pairs.  Accumulators of the tensor
+    core are truncated after every MMA, so no run may exceed 8,192 rows."""
+    n, k = 400_000, 2_048
+    g = torch.Generator(device="cuda")
+    g.manual_seed(77)
+    X = torch.rand((n, k), generator=g, device="cuda") + 0.5
+    F = G.grass_fim(X)
+    cols = [0, 1, 127, 128, 1_000, 2_047]
+    ref, _ = oracle_mod.fim(np.ascontiguousarray(X[:, cols].cpu().numpy()))
+    got = F[cols][:, cols].cpu().numpy().astype(np.float64)
+    assert (np.abs(got - ref) / np.abs(ref)).max() <= 1e-4
+    del X, F
+    torch.cuda.empty_cache()
+
+    B, T, d, kk, k_out, L = 256, 32_768, 64, 64, 4_096, 4
+    A = (torch.rand((B, T, d), generator=g, device="cuda") + 0.5).to(torch.bfloat16)
+    Gt = (torch.rand((B, T, d), generator=g, device="cuda") + 0.5).to(torch.bfloat16)
+    ident = np.arange(kk, dtype=np.uint32)
+    dev_ident = G.mask_to_device(ident)
+    layers = [dict(A=A, G=Gt, mask_in=dev_ident, mask_out=dev_ident, k=k_out, s=1, seed=900 + l, out_offset=l * k_out)
+              for l in range(L)]
+    ws = torch.empty(G.factgrass_grouped_workspace_bytes(L), dtype=torch.uint8, device="cuda")
+    out = torch.empty((B, L * k_out), device="cuda")
+    G.factgrass_compress_grouped(G.GroupedLayers(layers), out, ws)
+    for (b, l) in [(0, 0), (255, 3)]:
+        ref, absum = oracle_mod.factgrass(W.bits_of(A[b:b + 1]), W.bits_of(Gt[b:b + 1]), ident, ident, k_out, 1, 900 + l)
+        got = out[b, l * k_out:(l + 1) * k_out].cpu().numpy().astype(np.float64)
+        # a bin holds entries of both signs: compare against the sum of magnitudes
+        used = absum[0] > 0
+        assert (np.abs(got - ref[0])[used] / absum[0][used]).max() <= 1e-4
+        assert np.all(got[~used] == 0.0)
