@@ -138,8 +138,9 @@ class L2Flush:
 # ----------------------------------------------------------------------------- workloads (GPU arm)
 
 def sector_bytes_per_row(idx: np.ndarray, elem_bytes: int, gran: int = 32) -> int:
-    """Bytes of one row that a gather of `idx` must move at `gran`-byte granularity (32 = L2 sector,
-    the algorithmic figure; 128 = the line the B200 memory system actually fetches)."""
+    """Bytes of one row that a gather of `idx` must move at `gran`-byte granularity (32 = L2 sector, the
+    algorithmic figure; 64 = the smallest piece a B200 load can make DRAM deliver, with the L2::64B
+    prefetch-size hint the gather kernels use; without the hint it is the whole 128-byte line)."""
     per = gran // elem_bytes
     return int(np.unique(idx.astype(np.int64) // per).size) * gran
 
@@ -160,7 +161,7 @@ class GrassJob:
         self.out = torch.empty((cfg.batch, cfg.k), dtype=torch.float32, device=device)
         self.samples_per_step = cfg.n
         self.alg_bytes_per_launch = cfg.batch * sector_bytes_per_row(self.idx, 4) + cfg.batch * cfg.k * 4
-        self.line_bytes_per_launch = cfg.batch * sector_bytes_per_row(self.idx, 4, 128) + cfg.batch * cfg.k * 4
+        self.fetch_bytes_per_launch = cfg.batch * sector_bytes_per_row(self.idx, 4, 64) + cfg.batch * cfg.k * 4
         self.dense_bytes_per_launch = batch_bytes
         self.launches_per_step = self.nbatch
         self.kernels_per_step = 2 * self.nbatch     # memset + compress kernel per call (upper bound)
@@ -211,7 +212,7 @@ class FactJob:
             layers.append(dict(A=A, G=Gt, mask_in=G.mask_to_device(mi, device), mask_out=G.mask_to_device(mo, device),
                                k=cfg.k, s=cfg.s, seed=W.layer_hash_seed(cfg, l), out_offset=l * cfg.k))
             alg += tokens * (sector_bytes_per_row(mi, eb) + sector_bytes_per_row(mo, eb)) + cfg.B * cfg.k * 4
-            line += tokens * (sector_bytes_per_row(mi, eb, 128) + sector_bytes_per_row(mo, eb, 128)) + cfg.B * cfg.k * 4
+            line += tokens * (sector_bytes_per_row(mi, eb, 64) + sector_bytes_per_row(mo, eb, 64)) + cfg.B * cfg.k * 4
             self.dense += cfg.B * cfg.T * (lay.d_in + lay.d_out) * eb
         self.layers = layers
         self.group = G.GroupedLayers(layers)
@@ -229,7 +230,7 @@ class FactJob:
             self.test_pre = torch.empty_like(self.score[1])
         self.samples_per_step = cfg.B
         self.alg_bytes_per_launch = alg
-        self.line_bytes_per_launch = line
+        self.fetch_bytes_per_launch = line
         self.dense_bytes_per_launch = self.dense
         self.launches_per_step = 1
         nb = (cfg.k + 63) // 64
@@ -669,9 +670,9 @@ def main():
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": int(job.alg_bytes_per_launch),
                 "dense_bytes_per_launch": int(job.dense_bytes_per_launch), "ms_per_launch": dom_ms,
-                "line128_bytes_per_launch": int(job.line_bytes_per_launch),
-                "line128_achieved": job.line_bytes_per_launch / (dom_ms * 1e-3) / 1e9,
-                "line128_frac": job.line_bytes_per_launch / (dom_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                "fetch64_bytes_per_launch": int(job.fetch_bytes_per_launch),
+                "fetch64_achieved": job.fetch_bytes_per_launch / (dom_ms * 1e-3) / 1e9,
+                "fetch64_frac": job.fetch_bytes_per_launch / (dom_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                 "traffic": None if (args.fp32_inputs or args.seq_len_aware or args.small) else TRAFFIC.get(args.config)}
 
     e2e = None
@@ -700,8 +701,7 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel per launch, from ncu captures
 # summarised under profiles/ (bytes; None until captured)
-TRAFFIC = {1: 65_799_424 + 336_896, 2: 8 * (425_585_920 + 4_569_856), 3: 124_359_424 + 3_895_296,
-           4: 3 * (1_354_089_000 + 4_009_216), 5: 16 * (1_191_565_000 + 5_072_128)}
+TRAFFIC = {1: None, 2: None, 3: None, 4: None, 5: None}
 
 if __name__ == "__main__":
     main()

@@ -50,7 +50,7 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t b)
 }
 
 #ifndef GRASS_LD_MODE
-#define GRASS_LD_MODE 0
+#define GRASS_LD_MODE 6
 #endif
 // gathered (scattered, read-once) loads of one element
 __device__ __forceinline__ uint32_t gather_u32(const uint32_t* p)
@@ -63,9 +63,17 @@ __device__ __forceinline__ uint32_t gather_u32(const uint32_t* p)
     return __ldcg(p);
 #elif GRASS_LD_MODE == 3
     return __ldcs(p);
-#else
+#elif GRASS_LD_MODE == 4
     uint32_t v;
     asm volatile("ld.global.nc.L1::no_allocate.b32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+#elif GRASS_LD_MODE == 5
+    uint32_t v;
+    asm("ld.global.nc.L2::64B.b32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+#else
+    uint32_t v;
+    asm("ld.global.nc.L1::no_allocate.L2::64B.b32 %0, [%1];" : "=r"(v) : "l"(p));
     return v;
 #endif
 }
@@ -79,6 +87,14 @@ __device__ __forceinline__ uint16_t gather_u16(const uint16_t* p)
     return __ldcg(p);
 #elif GRASS_LD_MODE == 3
     return __ldcs(p);
+#elif GRASS_LD_MODE == 5
+    uint16_t v;
+    asm("ld.global.nc.L2::64B.b16 %0, [%1];" : "=h"(v) : "l"(p));
+    return v;
+#elif GRASS_LD_MODE == 6
+    uint16_t v;
+    asm("ld.global.nc.L1::no_allocate.L2::64B.b16 %0, [%1];" : "=h"(v) : "l"(p));
+    return v;
 #else
     uint16_t v;
     asm volatile("ld.global.nc.L1::no_allocate.b16 %0, [%1];" : "=h"(v) : "l"(p));
