@@ -53,12 +53,16 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 def build_microbench() -> str:
-    """Compile the stand-alone DRAM fetch-granularity microbenchmark (not part of the library)."""
-    out = os.path.join(HERE, "_build", "fetch_granularity")
-    os.makedirs(os.path.dirname(out), exist_ok=True)
-    subprocess.check_call([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-o", out,
-                           os.path.join(CSRC, "microbench", "fetch_granularity.cu")])
-    return out
+    """Compile the stand-alone DRAM fetch-granularity microbenchmarks (not part of the library)."""
+    bdir = os.path.join(HERE, "_build")
+    os.makedirs(bdir, exist_ok=True)
+    outs = []
+    for name in ("fetch_granularity", "tma_box_granularity"):
+        out = os.path.join(bdir, name)
+        subprocess.check_call([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-o", out,
+                               os.path.join(CSRC, "microbench", name + ".cu")])
+        outs.append(out)
+    return " ".join(outs)
 
 
 if __name__ == "__main__":

@@ -52,7 +52,10 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t b)
 #ifndef GRASS_LD_MODE
 #define GRASS_LD_MODE 6
 #endif
-// gathered (scattered, read-once) loads of one element
+// Gathered (scattered, read-once) loads of one element.  On B200 a plain load of an untouched 128-byte line makes
+// DRAM deliver the whole line; the L2::64B prefetch-size hint limits the fetch to the 64-byte half that holds the
+// element (nothing fetches less), which is what a sparse mask wants.  L1::no_allocate: the data are used once.
+// GRASS_LD_MODE selects other load forms for comparison builds.
 __device__ __forceinline__ uint32_t gather_u32(const uint32_t* p)
 {
 #if GRASS_LD_MODE == 0
