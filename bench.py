@@ -342,8 +342,10 @@ def time_job(job, steps, warmup, world, device):
 # ----------------------------------------------------------------------------- end-to-end (host buffers)
 
 def e2e_job(cfg_id, job, steps, warmup, world, device, G, W):
-    """The same metric through the host-buffer API: every step copies the step's inputs from pinned
-    host memory to the device, compresses, and reads the result back."""
+    """The same metric through the host-buffer API with the inputs in pinned host memory, the result read back
+    every step.  Two legs: "in place" (the API's default for pinned inputs: the kernels gather the masked elements
+    from host memory across the bus, so only the 64-byte pieces the masks touch are moved) and "staged" (every
+    input byte is copied to the device first).  The line's `e2e` is the in-place leg; the staged one rides along."""
     from paper_2505_18976_b200 import host_api
     cfg = job.cfg
     if cfg_id in (1, 2):
@@ -356,8 +358,12 @@ def e2e_job(cfg_id, job, steps, warmup, world, device, G, W):
         d2h = cfg.n * cfg.k * 4
         note = f"{cfg.n // rows} chunk copies of {rows} rows from one pinned staging buffer"
 
-        def run():
-            host_api.grass_compress_host(chunks, job.idx, cfg.k, cfg.s, cfg.hash_seed, out_host=out_host, device=device)
+        pieces = (job.fetch_bytes_per_launch - cfg.batch * cfg.k * 4) * job.launches_per_step
+        in_place = host_api.grass_in_place(chunks, job.idx)
+
+        def run(zero_copy):
+            host_api.grass_compress_host(chunks, job.idx, cfg.k, cfg.s, cfg.hash_seed, out_host=out_host, device=device,
+                                         zero_copy=zero_copy)
     else:
         # pinned copies of the first block's layers; later blocks of the same shape reuse those host
         # tensors (the bytes copied per step are those of the whole model)
@@ -387,24 +393,42 @@ def e2e_job(cfg_id, job, steps, warmup, world, device, G, W):
             h2d += (score_host[0].numel() + score_host[1].numel()) * 4
             d2h += cfg.score_n_train * cfg.score_n_test * 4
 
-        def run():
-            host_api.factgrass_compress_host(groups, cfg.B, cfg.T, cfg.out_dim, out_host=out_host, device=device)
+        score_bytes = (score_host[0].numel() + score_host[1].numel()) * 4 if score_host else 0
+        pieces = job.fetch_bytes_per_launch - cfg.B * cfg.out_dim * 4 + score_bytes
+        in_place = host_api.factgrass_in_place(groups)
+
+        def run(zero_copy):
+            host_api.factgrass_compress_host(groups, cfg.B, cfg.T, cfg.out_dim, out_host=out_host, device=device,
+                                             zero_copy=zero_copy)
             if score_host:
                 host_api.grass_score_host(score_host[0], score_host[1], device=device)
 
-    for _ in range(max(1, min(warmup, 2))):
-        run()
-    torch.cuda.synchronize()
-    barrier(world)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        run()
-    e1.record()
-    torch.cuda.synchronize()
-    ms = max_over_ranks(e0.elapsed_time(e1) / steps, world, device)
-    return {"value": world * job.samples_per_step / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
-            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps, "staging": note}
+    def leg(zero_copy):
+        for _ in range(max(1, min(warmup, 2))):
+            run(zero_copy)
+        torch.cuda.synchronize()
+        barrier(world)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            run(zero_copy)
+        e1.record()
+        torch.cuda.synchronize()
+        return max_over_ranks(e0.elapsed_time(e1) / steps, world, device)
+
+    ms_staged = leg(False)
+    ms_in_place = leg(True)
+    ms_default = leg(None)                 # what the call does when left to choose
+    per_s = world * job.samples_per_step
+    return {"value": per_s / (ms_default * 1e-3), "unit": UNIT, "ms_per_step": ms_default,
+            "h2d_bytes_per_step": int(pieces if in_place else h2d), "d2h_bytes_per_step": int(d2h), "steps": steps,
+            "path": ("in place: the kernels gather from the pinned host inputs; h2d = 64-byte pieces the masks touch "
+                     "(host count)" + (" + the score operands, which are copied" if cfg_id == 5 else ""))
+                    if in_place else "staged: every input byte is copied to the device (" + note + ")",
+            "host_input_bytes_per_step": int(h2d),
+            "staged": {"value": per_s / (ms_staged * 1e-3), "ms_per_step": ms_staged, "h2d_bytes_per_step": int(h2d)},
+            "in_place": {"value": per_s / (ms_in_place * 1e-3), "ms_per_step": ms_in_place,
+                         "h2d_bytes_per_step": int(pieces)}}
 
 
 # ----------------------------------------------------------------------------- CPU oracle arm

@@ -12,6 +12,10 @@
  * Conventions (all calls):
  *   - Pointers are DEVICE pointers unless the parameter is marked "host".  The caller owns every
  *     buffer; the library allocates nothing and keeps no state between calls.
+ *   - The gathered inputs (g of grass_compress / grass_mask, A and G of the factgrass / factmask calls) may
+ *     also be page-locked host memory that the device can address (cudaHostAlloc, cudaHostRegister): the
+ *     kernels then read the masked elements in place across the bus, 64 bytes per touched piece, which for a
+ *     sparse mask moves far less than copying the inputs would.  Every other buffer is device memory.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work is
  *     enqueued on it and the call returns without synchronising, except where stated.
  *   - Output buffers are OVERWRITTEN (the call zeroes them itself where its kernels accumulate).

@@ -137,18 +137,32 @@ def _need_cuda(*ts) -> None:
             raise ValueError("device tensors required (the library has no CPU path)")
 
 
+def _need_device_readable(*ts) -> None:
+    """Inputs the kernels only gather from: device tensors, or page-locked host tensors (which the device
+    addresses directly; the kernels then pull the masked elements across the bus)."""
+    for t in ts:
+        if t is not None and not (t.is_cuda or t.is_pinned()):
+            raise ValueError("device or pinned host tensors required (the library has no CPU path)")
+
+
+def _compute_device(t: torch.Tensor) -> torch.device:
+    return t.device if t.is_cuda else torch.device("cuda", torch.cuda.current_device())
+
+
 def grass_compress(g: torch.Tensor, idx: Optional[torch.Tensor], k: int, s: int, seed: int,
                    out: Optional[torch.Tensor] = None, p: Optional[int] = None,
                    dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
     """out[i] = SJLT_{k,s,seed}(g[i, idx]) for the rows of g (n x ld, fp32 or bf16).
-    idx: uint32/int32 CUDA tensor of ascending coordinates, or None for the identity mask."""
-    _need_cuda(g, idx, out, dev_status)
+    idx: uint32/int32 CUDA tensor of ascending coordinates, or None for the identity mask.
+    g may be a pinned host tensor: the kernel then reads the masked elements in place, across the bus."""
+    _need_device_readable(g)
+    _need_cuda(idx, out, dev_status)
     assert g.dim() == 2 and g.stride(1) == 1
     n, ld = g.shape[0], g.stride(0) if g.shape[0] > 1 else g.shape[1]
     p = g.shape[1] if p is None else p
     kprime = p if idx is None else idx.numel()
     if out is None:
-        out = torch.empty((n, k), dtype=torch.float32, device=g.device)
+        out = torch.empty((n, k), dtype=torch.float32, device=_compute_device(g))
     assert out.dtype == torch.float32 and out.stride(1) == 1
     spec = SjltSpec(k, s, seed & 0xFFFFFFFFFFFFFFFF)
     _check(lib().grass_compress(_ptr(g), _dt(g), n, p, ld, _ptr(idx), kprime, ctypes.byref(spec), _ptr(out),
@@ -213,12 +227,14 @@ class GroupedLayers:
     """Host-side descriptor table for factgrass_compress_grouped; keeps the tensors alive."""
 
     def __init__(self, layers: Sequence[dict]):
-        """layers: dicts with A, G, mask_in, mask_out (CUDA tensors), k, s, seed, out_offset."""
+        """layers: dicts with A, G (CUDA tensors, or pinned host tensors read in place), mask_in, mask_out (CUDA
+        tensors), k, s, seed, out_offset."""
         self.keep = list(layers)
         self.L = len(layers)
         self.array = (FactgrassLayer * max(self.L, 1))()
         for i, l in enumerate(layers):
-            _need_cuda(l["A"], l["G"], l["mask_in"], l["mask_out"])
+            _need_device_readable(l["A"], l["G"])
+            _need_cuda(l["mask_in"], l["mask_out"])
             e = self.array[i]
             e.A, e.G = l["A"].data_ptr(), l["G"].data_ptr()
             e.mask_in, e.mask_out = l["mask_in"].data_ptr(), l["mask_out"].data_ptr()

@@ -86,3 +86,16 @@ def test_oracle_and_cuda_path_share_no_code():
         if f.endswith((".py", ".c", ".h")):
             src = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2505_18976_b200" not in src and "grass.h" not in src and "libgrass_b200" not in src
+
+
+def test_host_api_chooses_in_place_gather_only_for_sparse_masks():
+    """At 64-byte granularity a mask of every 64th fp32 coordinate touches a quarter of the pieces, a mask of every
+    4th coordinate touches all of them; unpinned inputs are always staged."""
+    import torch
+    from paper_2505_18976_b200 import host_api
+    assert host_api.touched_fraction(np.arange(0, 4096, 64), 4096, 4) == pytest.approx(0.25)
+    assert host_api.touched_fraction(np.arange(0, 4096, 4), 4096, 4) == 1.0
+    assert host_api.touched_fraction(np.array([0, 1, 31, 32]), 64, 2) == 1.0
+    g = torch.zeros((2, 4096))
+    assert not host_api.grass_in_place([g], np.arange(0, 4096, 64))          # not pinned
+    assert not host_api.grass_in_place([g], None)
