@@ -96,3 +96,31 @@ def test_grass_score_host(G, W, oracle_mod):
     sc = host_api.grass_score_host(_pinned(tr), _pinned(te))
     ref, absum = oracle_mod.score(tr.numpy(), te.numpy())
     check_close(sc.numpy(), ref, absum, TOL_F32, 140, what="host score")
+
+
+def test_config4_block_in_place_matches_device_resident(G, W, oracle_mod):
+    """One GPT-2-small block of config 4 (4 layers, 16 x 1,024 tokens) gathered from pinned host memory: same
+    results as from device memory up to the order of the atomic adds, and parity with the oracle on one layer."""
+    from paper_2505_18976_b200 import host_api
+    c = W.CONFIG4
+    dev_layers, host_layers = [], []
+    for l in range(4):
+        A, Gt = W.layer_io(c, l, device="cuda")
+        s_in, s_out = W.layer_mask_seeds(c, l)
+        mi = G.grass_random_mask_host(c.layers[l].d_in, c.kin, s_in)
+        mo = G.grass_random_mask_host(c.layers[l].d_out, c.kout, s_out)
+        common = dict(k=c.k, s=c.s, seed=W.layer_hash_seed(c, l), out_offset=l * c.k)
+        dev_layers.append(dict(A=A, G=Gt, mask_in=G.mask_to_device(mi), mask_out=G.mask_to_device(mo), **common))
+        host_layers.append(dict(A=_pinned(A.cpu()), G=_pinned(Gt.cpu()), mask_in=mi, mask_out=mo, **common))
+    assert host_api.factgrass_in_place([host_layers])
+    out_dev = torch.empty((c.B, 4 * c.k), device="cuda")
+    ws = torch.empty(G.factgrass_grouped_workspace_bytes(4), dtype=torch.uint8, device="cuda")
+    G.factgrass_compress_grouped(G.GroupedLayers(dev_layers), out_dev, ws)
+    out_host = host_api.factgrass_compress_host([host_layers], c.B, c.T, 4 * c.k)
+    a, b = out_dev.cpu().numpy().astype(np.float64), out_host.numpy().astype(np.float64)
+    assert np.abs(a - b).max() <= 1e-5 * np.abs(a).max()
+    l = 2
+    ref, absum = oracle_mod.factgrass(W.bits_of(dev_layers[l]["A"]), W.bits_of(dev_layers[l]["G"]),
+                                      host_layers[l]["mask_in"], host_layers[l]["mask_out"], c.k, c.s,
+                                      W.layer_hash_seed(c, l))
+    check_close(b[:, l * c.k:(l + 1) * c.k], ref, absum, TOL_BF16, c.T + 64, eps=EPS_TC, what="config 4 block, in place")
