@@ -21,6 +21,12 @@ namespace cg = cooperative_groups;
 namespace grass {
 
 constexpr int kThreads = 256;
+// Dense rows with many zeros: the non-zero entries of a warp's round of loads are first compacted into a small
+// per-warp queue in shared memory, so that every lane hashes a non-zero (the cost of the projection follows the
+// non-zeros, Section 3.1) instead of the whole warp waiting on the lanes that hold one.
+constexpr int kQueueCap = 128;                                  // entries per warp; fuller rounds are hashed in place
+// an entry = the value and a 16-bit key: (position within the round) * 8 + sample of the CTA
+constexpr int kQueueBytes = (kThreads / 32) * kQueueCap * (int)(sizeof(float) + sizeof(uint16_t));
 
 // four consecutive elements of a row with one vector load (16 bytes of fp32, 8 bytes of bf16)
 __device__ __forceinline__ void load4(const float* p, float (&v)[4])
@@ -38,7 +44,7 @@ __device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&v)[4])
 // DENSE: identity mask on vector-aligned rows (plain SJLT, the k' = p case of Section 3.3.1).  Rows are then
 // streamed with vector loads, four consecutive positions per thread, and S > 1 samples share each hash.
 template <typename T, int S, int U, bool S1, bool DENSE>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, DENSE ? 4 : 0)
 grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
                       const uint32_t* __restrict__ idx, int64_t kprime, uint32_t k, uint32_t s,
                       uint64_t seed, float scale, float* __restrict__ out, int64_t ld_out,
@@ -63,7 +69,16 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
     bool bad = false;
     if constexpr (DENSE) {
         constexpr int UD = S >= 8 ? 1 : 8 / S;     // vector loads per sample in flight per thread (8 in all)
-        for (int64_t jb = j0 + (int64_t)tid * 4; jb < j1; jb += (int64_t)kThreads * 4 * UD) {
+        const int lane = tid & 31, warp = tid >> 5;
+        // this warp's queue, behind the bins (8-byte aligned)
+        unsigned char* qbase = reinterpret_cast<unsigned char*>(bins) +
+                               (use_smem ? (((size_t)S * k * sizeof(float) + 7) & ~(size_t)7) : 0);
+        float* qval = reinterpret_cast<float*>(qbase) + warp * kQueueCap;
+        uint16_t* qkey = reinterpret_cast<uint16_t*>(qbase + (kThreads / 32) * kQueueCap * sizeof(float)) + warp * kQueueCap;
+        static_assert(kThreads * 4 * UD * 8 <= 65536 && S <= 8, "queue key is 16 bits");
+        // the trip count is the same for every thread (the warp votes below); positions beyond j1 load as zeros
+        for (int64_t round0 = j0; round0 < j1; round0 += (int64_t)kThreads * 4 * UD) {
+            const int64_t jb = round0 + (int64_t)tid * 4;
             float v[UD][S][4];
 #pragma unroll
             for (int u = 0; u < UD; ++u) {
@@ -78,6 +93,64 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
                             v[u][si][e] = (si < ns && j + e < j1) ? elem<T>::load(rows[si] + j + e) : 0.0f;
                     }
                 }
+            }
+            // Non-zeros of this round: per lane, then over the warp.  The first vector of every lane is counted
+            // first: where that sample already says the round is too full for the queue, the exact count is skipped.
+            bool queue = false;
+            uint32_t cnt = 0, total = 0;
+#pragma unroll
+            for (int si = 0; si < S; ++si)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) cnt += (v[0][si][e] != 0.0f) ? 1u : 0u;
+            if (__reduce_add_sync(0xFFFFFFFFu, cnt) * UD <= 2u * kQueueCap) {
+#pragma unroll
+                for (int u = 1; u < UD; ++u)
+#pragma unroll
+                    for (int si = 0; si < S; ++si)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) cnt += (v[u][si][e] != 0.0f) ? 1u : 0u;
+                total = __reduce_add_sync(0xFFFFFFFFu, cnt);
+                if (total == 0) continue;
+                queue = total <= (uint32_t)kQueueCap;
+            }
+            if (queue) {
+                uint32_t incl = cnt;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    if (lane >= d) incl += t;
+                }
+                uint32_t at = incl - cnt;
+#pragma unroll
+                for (int u = 0; u < UD; ++u)
+#pragma unroll
+                    for (int si = 0; si < S; ++si)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float x = v[u][si][e];
+                            if (x != 0.0f) {
+                                qval[at] = x;
+                                qkey[at] = (uint16_t)(((tid * 4 + u * kThreads * 4 + e) << 3) | si);
+                                ++at;
+                            }
+                        }
+                __syncwarp();
+                for (uint32_t q = lane; q < total; q += 32) {
+                    const uint32_t key = qkey[q];
+                    const uint32_t si = key & 7u;
+                    const float x = qval[q];
+                    const uint64_t pos = (uint64_t)(round0 + (int64_t)(key >> 3));
+                    const uint32_t draws = S1 ? 1u : s;
+                    for (uint32_t r = 0; r < draws; ++r) {
+                        const uint64_t h = sjlt_hash_counter(seed, S1 ? (pos + 1) : (pos * s + r + 1));
+                        const uint32_t b = sjlt_bucket(h, k);
+                        const float sx = S1 ? sjlt_signed(h, x) : sjlt_signed(h, x) * scale;
+                        if (use_smem) atomicAdd(&bins[si * k + b], sx);
+                        else atomicAdd(out + (i0 + si) * ld_out + b, sx);
+                    }
+                }
+                __syncwarp();       // the queue is rewritten in the next round
+                continue;
             }
 #pragma unroll
             for (int u = 0; u < UD; ++u) {
@@ -272,7 +345,8 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
     if (pl.dense) j_per_cta = (j_per_cta + 3) / 4 * 4;      // vector loads start on multiples of four positions
     // 0: one CTA owns the row, plain stores; 1: global reductions into a zeroed row; 2: cluster reduction
     const int accumulate = pl.cluster ? 2 : ((pl.jsplit > 1 || !pl.use_smem) ? 1 : 0);
-    const size_t smem = pl.use_smem ? (size_t)S * sp.k * sizeof(float) : 0;
+    size_t smem = pl.use_smem ? (size_t)S * sp.k * sizeof(float) : 0;
+    if (pl.dense) smem = ((smem + 7) & ~(size_t)7) + kQueueBytes;      // the warps' non-zero queues
     const float scale = 1.0f / sqrtf((float)sp.s);
     auto launch = [&](auto kern) -> grass_status {
         if (smem > 48 * 1024) {

@@ -117,6 +117,22 @@ def test_grass_compress_identity_mask_and_stride(G, W, oracle_mod):
     _grass_case(G, W, oracle_mod, 5, 9_001, 9_001, 100, ld=9_016, identity=True)
 
 
+@pytest.mark.parametrize("zero_prob", [0.0, 0.5, 0.9, 0.99, 0.999])
+def test_plain_sjlt_over_input_sparsity(G, W, oracle_mod, monkeypatch, zero_prob):
+    """Identity mask on vector-aligned rows: rounds of loads with few non-zeros go through the per-warp queue, fuller
+    ones are hashed in place; one and two samples per CTA, s = 1 and 2, fp32 and bf16, a ragged tail, an odd k,
+    and a k whose bins do not fit in shared memory."""
+    for S in (1, 2):
+        monkeypatch.setenv("GRASS_COMPRESS_S", str(S))
+        _grass_case(G, W, oracle_mod, 9, 131_072, 131_072, 4_096, identity=True, zero_prob=zero_prob)
+        _grass_case(G, W, oracle_mod, 5, 40_004, 40_004, 777, s=2, identity=True, zero_prob=zero_prob)
+        _grass_case(G, W, oracle_mod, 4, 33_000, 33_000, 512, identity=True, zero_prob=zero_prob, dtype=torch.bfloat16)
+    monkeypatch.delenv("GRASS_COMPRESS_S")
+    _grass_case(G, W, oracle_mod, 3, 70_000, 70_000, 60_000, identity=True, zero_prob=zero_prob)
+    monkeypatch.setenv("GRASS_COMPRESS_JSPLIT", "5")
+    _grass_case(G, W, oracle_mod, 3, 50_000, 50_000, 300, identity=True, zero_prob=zero_prob)
+
+
 def test_grass_compress_bf16_input(G, W, oracle_mod):
     _grass_case(G, W, oracle_mod, 12, 100_000, 10_000, 1_024, dtype=torch.bfloat16)
 
