@@ -738,7 +738,7 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel per launch, from ncu captures
 # summarised under profiles/ (bytes; None until captured)
-TRAFFIC = {1: 58_786_048 + 329_728, 2: 8 * (239_955_712 + 3_990_016), 3: 101_295_360 + 3_341_312,
+TRAFFIC = {1: 58_786_304 + 489_984, 2: 8 * (239_941_632 + 3_357_184), 3: 101_295_360 + 3_341_312,
            4: 3 * (1_044_521_000 + 3_736_576), 5: 16 * (729_330_432 + 4_238_848)}
 
 if __name__ == "__main__":
