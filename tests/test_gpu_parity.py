@@ -285,6 +285,22 @@ def test_factgrass_token_chunking(G, W, oracle_mod, monkeypatch, chunk):
     _fact_case(G, W, oracle_mod, _fact_cfg(W, T=250, kin=64, kout=64, k=512))
 
 
+@pytest.mark.parametrize("tile", [64, 128])
+def test_factgrass_seeded_shape_sweep(G, W, oracle_mod, monkeypatch, tile):
+    """Seeded random shapes: layer widths, mask sizes around the 64 / 128 tile edges, token counts that end inside a
+    32-token stage, output lengths on both sides of the block size, one or two draws, bf16 and fp32 factors."""
+    monkeypatch.setenv("FACTGRASS_TILE", str(tile))
+    rng = np.random.default_rng(1234 + tile)
+    for case in range(10):
+        d_in, d_out = int(rng.integers(8, 700)), int(rng.integers(8, 700))
+        kin = int(min(d_in, rng.choice([1, 7, 63, 64, 65, 127, 128, 129, 200])))
+        kout = int(min(d_out, rng.choice([1, 9, 63, 64, 65, 127, 128, 129, 150])))
+        cfg = _fact_cfg(W, layers=(W.LinearLayer("l", d_in, d_out),), B=int(rng.integers(1, 5)),
+                        T=int(rng.integers(1, 260)), kin=kin, kout=kout, k=int(rng.integers(1, 3 * kin * kout + 2)),
+                        s=int(rng.choice([1, 1, 2])), data_seed=300 + case, mask_seed=case, hash_seed=5 * case + 1)
+        _fact_case(G, W, oracle_mod, cfg, dtype=torch.float32 if case % 3 == 2 else torch.bfloat16)
+
+
 def test_factgrass_scaled_configs(G, W, oracle_mod):
     c3 = dataclasses.replace(W.CONFIG3, B=4, T=256)
     _fact_case(G, W, oracle_mod, c3)
