@@ -133,6 +133,21 @@ def test_plain_sjlt_over_input_sparsity(G, W, oracle_mod, monkeypatch, zero_prob
     _grass_case(G, W, oracle_mod, 3, 50_000, 50_000, 300, identity=True, zero_prob=zero_prob)
 
 
+def test_grass_compress_seeded_shape_sweep(G, W, oracle_mod):
+    """Seeded random shapes: row lengths, strides with a NaN tail beyond p, mask sizes from a handful to every
+    coordinate, output lengths from one bin to more bins than masked coordinates, one to three draws, both dtypes,
+    sparse and dense rows."""
+    rng = np.random.default_rng(4321)
+    for case in range(12):
+        p = int(rng.integers(40, 120_000))
+        kprime = int(rng.choice([1, 31, 33, p // 7 + 1, p // 2 + 1, p]))
+        identity = kprime == p and case % 2 == 0
+        _grass_case(G, W, oracle_mod, int(rng.integers(1, 20)), p, kprime, int(rng.integers(1, 6_000)),
+                    s=int(rng.choice([1, 1, 2, 3])), dtype=torch.bfloat16 if case % 4 == 1 else torch.float32,
+                    ld=p + 8 * int(rng.integers(0, 3)), identity=identity, zero_prob=float(rng.choice([0.0, 0.7, 0.97])),
+                    seed=case, data_seed=50 + case)
+
+
 def test_grass_compress_bf16_input(G, W, oracle_mod):
     _grass_case(G, W, oracle_mod, 12, 100_000, 10_000, 1_024, dtype=torch.bfloat16)
 
