@@ -175,13 +175,14 @@ def factgrass_compress(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, 
                        k: int, s: int, seed: int, out: Optional[torch.Tensor] = None,
                        dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
     """One linear layer: out[b] = SJLT(vec(sum_t A[b,t,mask_in] (x) G[b,t,mask_out]))."""
-    _need_cuda(A, G, mask_in, mask_out, out, dev_status)
+    _need_device_readable(A, G)
+    _need_cuda(mask_in, mask_out, out, dev_status)
     assert A.is_contiguous() and G.is_contiguous() and A.dim() == 3 and G.dim() == 3
     B, T, d_in = A.shape
     d_out = G.shape[2]
     assert G.shape[:2] == (B, T) and A.dtype == G.dtype
     if out is None:
-        out = torch.empty((B, k), dtype=torch.float32, device=A.device)
+        out = torch.empty((B, k), dtype=torch.float32, device=_compute_device(A))
     spec = SjltSpec(k, s, seed & 0xFFFFFFFFFFFFFFFF)
     _check(lib().factgrass_compress(_ptr(A), _ptr(G), _dt(A), B, T, d_in, d_out, _ptr(mask_in), mask_in.numel(),
                                     _ptr(mask_out), mask_out.numel(), ctypes.byref(spec), _ptr(out),
@@ -206,14 +207,15 @@ def factgrass_compress_varlen(A: torch.Tensor, G: torch.Tensor, mask_in: torch.T
     """One linear layer, samples with their own sequence lengths.  A, G: token-major (rows, d) matrices
     (or (B, T_max, d) for a padded batch); sample b owns rows tok_begin[b] .. + tok_count[b] (int64 /
     int32 CUDA tensors; None = b * T_max / T_max)."""
-    _need_cuda(A, G, mask_in, mask_out, out, dev_status)
+    _need_device_readable(A, G)
+    _need_cuda(mask_in, mask_out, out, dev_status)
     assert A.is_contiguous() and G.is_contiguous()
     _check_token_arrays(tok_begin, tok_count, B)
     d_in, d_out = A.shape[-1], G.shape[-1]
     if tok_begin is None:
         assert A.numel() >= B * T_max * d_in and G.numel() >= B * T_max * d_out
     if out is None:
-        out = torch.empty((B, k), dtype=torch.float32, device=A.device)
+        out = torch.empty((B, k), dtype=torch.float32, device=_compute_device(A))
     spec = SjltSpec(k, s, seed & 0xFFFFFFFFFFFFFFFF)
     _check(lib().factgrass_compress_varlen(_ptr(A), _ptr(G), _dt(A), B, T_max, _ptr(tok_begin), _ptr(tok_count),
                                            d_in, d_out, _ptr(mask_in), mask_in.numel(), _ptr(mask_out),
@@ -314,14 +316,15 @@ def grass_score(train: torch.Tensor, test: torch.Tensor, out: Optional[torch.Ten
 
 def grass_mask(g: torch.Tensor, idx: torch.Tensor, out: Optional[torch.Tensor] = None, p: Optional[int] = None,
                dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """Stand-alone Mask: out[i, j] = g[i, idx[j]] as fp32."""
-    _need_cuda(g, idx, out, dev_status)
+    """Stand-alone Mask: out[i, j] = g[i, idx[j]] as fp32.  g may be a pinned host tensor (read in place)."""
+    _need_device_readable(g)
+    _need_cuda(idx, out, dev_status)
     assert g.dim() == 2 and g.stride(1) == 1
     n, ld = g.shape[0], g.stride(0) if g.shape[0] > 1 else g.shape[1]
     p = g.shape[1] if p is None else p
     kp = idx.numel()
     if out is None:
-        out = torch.empty((n, kp), dtype=torch.float32, device=g.device)
+        out = torch.empty((n, kp), dtype=torch.float32, device=_compute_device(g))
     _check(lib().grass_mask(_ptr(g), _dt(g), n, p, ld, _ptr(idx), kp, _ptr(out),
                             out.stride(0) if n > 1 else max(out.shape[1], kp), _ptr(dev_status), _stream()), "grass_mask")
     return out
@@ -330,7 +333,8 @@ def grass_mask(g: torch.Tensor, idx: torch.Tensor, out: Optional[torch.Tensor] =
 def factmask_compress(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, mask_out: torch.Tensor,
                       out: Optional[torch.Tensor] = None, dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
     """Factorised Mask of one linear layer: out[b, a*kout + c] = sum_t A[b,t,mask_in[a]] G[b,t,mask_out[c]]."""
-    _need_cuda(A, G, mask_in, mask_out, out, dev_status)
+    _need_device_readable(A, G)
+    _need_cuda(mask_in, mask_out, out, dev_status)
     assert A.is_contiguous() and G.is_contiguous() and A.dim() == 3 and G.dim() == 3 and A.dtype == G.dtype
     B, T, d_in = A.shape
     d_out = G.shape[2]
@@ -338,7 +342,7 @@ def factmask_compress(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, m
     kout = d_out if mask_out is None else mask_out.numel()
     kp = kin * kout
     if out is None:
-        out = torch.empty((B, kp), dtype=torch.float32, device=A.device)
+        out = torch.empty((B, kp), dtype=torch.float32, device=_compute_device(A))
     _check(lib().factmask_compress(_ptr(A), _ptr(G), _dt(A), B, T, d_in, d_out, _ptr(mask_in), kin,
                                    _ptr(mask_out), kout, _ptr(out),
                                    out.stride(0) if B > 1 else max(out.shape[1], kp), _ptr(dev_status), _stream()),

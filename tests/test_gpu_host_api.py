@@ -124,3 +124,23 @@ def test_config4_block_in_place_matches_device_resident(G, W, oracle_mod):
                                       host_layers[l]["mask_in"], host_layers[l]["mask_out"], c.k, c.s,
                                       W.layer_hash_seed(c, l))
     check_close(b[:, l * c.k:(l + 1) * c.k], ref, absum, TOL_BF16, c.T + 64, eps=EPS_TC, what="config 4 block, in place")
+
+
+def test_single_layer_and_mask_calls_read_pinned_inputs_in_place(G, W, oracle_mod):
+    """factgrass_compress, factmask_compress and grass_mask given pinned host tensors."""
+    gen = torch.Generator().manual_seed(5)
+    A = _pinned(torch.randn((2, 90, 200), generator=gen).to(torch.bfloat16))
+    Gt = _pinned((torch.randn((2, 90, 120), generator=gen) * 1e-2).to(torch.bfloat16))
+    mi, mo = oracle_mod.random_mask(200, 30, 1), oracle_mod.random_mask(120, 20, 2)
+    dmi, dmo = G.mask_to_device(mi), G.mask_to_device(mo)
+    out = G.factgrass_compress(A, Gt, dmi, dmo, 333, 1, 17)
+    assert out.is_cuda
+    ref, absum = oracle_mod.factgrass(W.bits_of(A), W.bits_of(Gt), mi, mo, 333, 1, 17)
+    check_close(out.cpu().numpy(), ref, absum, TOL_BF16, 90 + 64, eps=EPS_TC, what="pinned single layer")
+    blk = G.factmask_compress(A, Gt, dmi, dmo)
+    ref, absum = oracle_mod.factmask(W.bits_of(A), W.bits_of(Gt), mi, mo)
+    check_close(blk.cpu().numpy(), ref, absum, TOL_BF16, 90 + 8, eps=EPS_TC, what="pinned factorised mask")
+    g = _pinned(W.dense_gradients(3, 5_000, 0.5, "normal", 1.0, 8, device="cpu"))
+    idx = oracle_mod.random_mask(5_000, 400, 3)
+    mk = G.grass_mask(g, G.mask_to_device(idx))
+    assert np.array_equal(mk.cpu().numpy(), oracle_mod.mask(W.bits_of(g), idx))
