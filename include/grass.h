@@ -8,6 +8,7 @@
  *   factgrass_compress           SJLT_k o Mask_{k'_in (x) k'_out} for one linear layer (Section 3.3.2)
  *   factgrass_compress_grouped   the same for many layers in one launch
  *   grass_score                  all-pair inner products of compressed vectors (Section 2.1, attribute stage)
+ *   grass_to_bf16, grass_score_bf16   the same for a cache stored in bf16
  *
  * Conventions (all calls):
  *   - Pointers are DEVICE pointers unless the parameter is marked "host".  The caller owns every
@@ -211,6 +212,20 @@ grass_status factgrass_compress_grouped_static(const factgrass_layer* layers /*h
  */
 grass_status grass_score(const float* train, int64_t N, int64_t ld_train, const float* test, int64_t M,
                          int64_t ld_test, int64_t D, float* scores, int64_t ld_s, void* stream);
+
+/*
+ * The same scores for a cache kept in bf16 (half the bytes of the attribute stage's inputs; the paper does not
+ * fix the storage precision, this is an option beside the fp32 path):
+ *   grass_to_bf16     out[i*ld_out + j] = bf16(in[i*ld_in + j]), round to nearest even; n <= 65,535 rows per call.
+ *   grass_score_bf16  scores[i*ld_s + m] = <train[i, :], test[m, :]> for bf16 train (N x D) and test (M x D);
+ *                     products are exact in fp32, accumulation as in grass_score; scores fp32, overwritten.
+ *                     Bases must be 16-byte aligned and ld_train, ld_test multiples of 8 (the rows are read by
+ *                     TMA); anything else returns GRASS_ERR_UNSUPPORTED with nothing enqueued.
+ */
+grass_status grass_to_bf16(const float* in, int64_t n, int64_t k, int64_t ld_in, void* out /* bf16 */, int64_t ld_out,
+                           void* stream);
+grass_status grass_score_bf16(const void* train /* bf16 */, int64_t N, int64_t ld_train, const void* test /* bf16 */,
+                              int64_t M, int64_t ld_test, int64_t D, float* scores, int64_t ld_s, void* stream);
 
 /*
  * Projected Fisher information matrix (Section 2.1, cache stage step 2):

@@ -28,7 +28,7 @@ EXPORTS = ("grass_compress", "factgrass_compress", "factgrass_compress_grouped",
            "grass_fim", "grass_fim_factor", "grass_fim_apply", "grass_mask", "factmask_compress",
            "factmask_compress_grouped",
            "factgrass_grouped_workspace_bytes", "factgrass_compress_grouped_static", "grass_score", "grass_sjlt_table", "grass_validate_mask",
-           "grass_random_mask_host", "grass_status_string")
+           "grass_random_mask_host", "grass_status_string", "grass_to_bf16", "grass_score_bf16")
 
 
 class GrassError(RuntimeError):
@@ -81,6 +81,10 @@ def lib() -> ctypes.CDLL:
                                                         i64, vp, vp]
         L.grass_score.restype = st
         L.grass_score.argtypes = [vp, i64, i64, vp, i64, i64, i64, vp, i64, vp]
+        L.grass_score_bf16.restype = st
+        L.grass_score_bf16.argtypes = [vp, i64, i64, vp, i64, i64, i64, vp, i64, vp]
+        L.grass_to_bf16.restype = st
+        L.grass_to_bf16.argtypes = [vp, i64, i64, i64, vp, i64, vp]
         L.grass_mask.restype = st
         L.grass_mask.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, i64, vp, i64, vp, vp]
         L.factmask_compress.restype = st
@@ -311,6 +315,37 @@ def grass_score(train: torch.Tensor, test: torch.Tensor, out: Optional[torch.Ten
     _check(lib().grass_score(_ptr(train), N, train.stride(0) if N > 1 else D, _ptr(test), M,
                              test.stride(0) if M > 1 else D, D, _ptr(out), out.stride(0) if N > 1 else M,
                              _stream()), "grass_score")
+    return out
+
+
+def grass_to_bf16(x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Compressed vectors as bf16 (round to nearest even), for a cache at half the size."""
+    _need_cuda(x, out)
+    assert x.dtype == torch.float32 and x.dim() == 2 and x.stride(1) == 1
+    n, k = x.shape
+    if out is None:
+        out = torch.empty((n, k), dtype=torch.bfloat16, device=x.device)
+    assert out.dtype == torch.bfloat16 and out.stride(1) == 1
+    for r0 in range(0, n, 65_535):
+        r1 = min(n, r0 + 65_535)
+        _check(lib().grass_to_bf16(_ptr(x[r0:r1]), r1 - r0, k, x.stride(0) if n > 1 else k, _ptr(out[r0:r1]),
+                                   out.stride(0) if n > 1 else k, _stream()), "grass_to_bf16")
+    return out
+
+
+def grass_score_bf16(train: torch.Tensor, test: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """scores[i, m] = <train[i], test[m]> for bf16 vectors (fp32 scores)."""
+    _need_cuda(train, test, out)
+    assert train.dtype == torch.bfloat16 and test.dtype == torch.bfloat16
+    assert train.stride(1) == 1 and test.stride(1) == 1
+    N, D = train.shape
+    M = test.shape[0]
+    assert test.shape[1] == D
+    if out is None:
+        out = torch.empty((N, M), dtype=torch.float32, device=train.device)
+    _check(lib().grass_score_bf16(_ptr(train), N, train.stride(0) if N > 1 else D, _ptr(test), M,
+                                  test.stride(0) if M > 1 else D, D, _ptr(out), out.stride(0) if N > 1 else M,
+                                  _stream()), "grass_score_bf16")
     return out
 
 

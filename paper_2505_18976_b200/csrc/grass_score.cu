@@ -103,6 +103,18 @@ grass_score_kernel(const float* __restrict__ train, int64_t N, int64_t ld_train,
 grass_status launch_score_tc(const float* train, int64_t N, int64_t ld_train, const float* test, int64_t M,
                              int64_t ld_test, int64_t D, float* scores, int64_t ld_s, cudaStream_t st);
 bool score_tc_supported(const float* train, int64_t ld_train, const float* test, int64_t ld_test, int64_t D);
+grass_status launch_score_bf16(const void* train, int64_t N, int64_t ld_train, const void* test, int64_t M,
+                               int64_t ld_test, int64_t D, float* scores, int64_t ld_s, cudaStream_t st);
+bool score_bf16_supported(const void* train, int64_t ld_train, const void* test, int64_t ld_test, int64_t D);
+
+// fp32 -> bf16, round to nearest even, row by row
+__global__ void to_bf16_kernel(const float* __restrict__ in, int64_t n, int64_t k, int64_t ld_in,
+                               __nv_bfloat16* __restrict__ out, int64_t ld_out)
+{
+    const int64_t i = blockIdx.y;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < k; j += (int64_t)gridDim.x * blockDim.x)
+        out[i * ld_out + j] = __float2bfloat16_rn(in[i * ld_in + j]);
+}
 
 }  // namespace grass
 
@@ -123,4 +135,31 @@ extern "C" grass_status grass_score(const float* train, int64_t N, int64_t ld_tr
     grass::grass_score_kernel<<<grid, grass::SC_THREADS, 0, (cudaStream_t)stream>>>(
         train, N, ld_train, test, M, ld_test, D, scores, ld_s, vec_ok);
     return grass::launch_status();
+}
+
+extern "C" grass_status grass_to_bf16(const float* in, int64_t n, int64_t k, int64_t ld_in, void* out, int64_t ld_out,
+                                      void* stream)
+{
+    if (n < 0 || k < 0 || ld_in < k || ld_out < k) return GRASS_ERR_INVALID_ARG;
+    if (n == 0 || k == 0) return GRASS_OK;
+    if (!in || !out) return GRASS_ERR_INVALID_ARG;
+    if (n > 65535) return GRASS_ERR_UNSUPPORTED;
+    int64_t gx = (k + 1023) / 1024;
+    if (gx > 1024) gx = 1024;
+    dim3 grid((unsigned)gx, (unsigned)n);
+    grass::to_bf16_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(in, n, k, ld_in, (__nv_bfloat16*)out, ld_out);
+    return grass::launch_status();
+}
+
+extern "C" grass_status grass_score_bf16(const void* train, int64_t N, int64_t ld_train, const void* test, int64_t M,
+                                         int64_t ld_test, int64_t D, float* scores, int64_t ld_s, void* stream)
+{
+    if (N < 0 || M < 0 || D < 0 || ld_train < D || ld_test < D || ld_s < M) return GRASS_ERR_INVALID_ARG;
+    if (N == 0 || M == 0) return GRASS_OK;
+    if (!scores || (D > 0 && (!train || !test))) return GRASS_ERR_INVALID_ARG;
+    if (D == 0)
+        return grass::cuda_ok(cudaMemset2DAsync(scores, (size_t)ld_s * sizeof(float), 0, (size_t)M * sizeof(float),
+                                                (size_t)N, (cudaStream_t)stream));
+    if (!grass::score_bf16_supported(train, ld_train, test, ld_test, D)) return GRASS_ERR_UNSUPPORTED;
+    return grass::launch_score_bf16(train, N, ld_train, test, M, ld_test, D, scores, ld_s, (cudaStream_t)stream);
 }

@@ -360,6 +360,209 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// The same contraction for vectors already stored as bf16 (a cache of compressed gradients at half the size):
+// no split is needed, so there are no producer warps at all.  TMA writes the bf16 tiles (128 rows x 32 k-values,
+// 64-byte swizzle) straight into the K-major operand layout the tensor core reads; per CTA one warp issues the
+// loads, one forwards "my tiles have landed" to the leader CTA's barriers, one thread of the leader issues the
+// MMAs (one product per 16 k-values), four warps drain the accumulator.
+#ifndef GRASS_H_STAGES
+#define GRASS_H_STAGES 8
+#endif
+constexpr int H_STAGES = GRASS_H_STAGES;
+constexpr int H_A_BYTES = BM * BK * 2;                   // this CTA's 128 train rows x 32 k-values of bf16: 8 KB
+constexpr int H_B_BYTES = BNH * BK * 2;                  // this CTA's half of the test rows: 8 KB
+constexpr int H_STAGE_BYTES = H_A_BYTES + H_B_BYTES;
+constexpr int H_BOX_ROWS = 32;                           // rows per TMA box
+constexpr int H_BOXES = BM / H_BOX_ROWS;                 // boxes per operand tile
+constexpr int H_EPI_WARPS = 4;
+constexpr int H_THREADS = (H_EPI_WARPS + 3) * 32;        // + MMA / tensor-memory warp, TMA warp, forwarding warp
+constexpr uint32_t H_TMEM_COLS = 256;                    // one fp32 accumulator of BN columns
+static_assert(H_STAGE_BYTES % 1024 == 0 && H_A_BYTES % 512 == 0, "operand tiles stay 512-byte aligned");
+static_assert(H_STAGES <= 32 && 2 * H_BOXES <= 32 && BM == BNH && (H_BOX_ROWS * ROW_BYTES) % 512 == 0,
+              "one stage and one box per lane");
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(H_THREADS, 1)
+grass_score_bf16_kernel(const __grid_constant__ CUtensorMap map_train, const __grid_constant__ CUtensorMap map_test,
+                        int64_t N, int64_t M, int64_t D, int64_t kt_split, float* __restrict__ scores, int64_t ld_s,
+                        int out_vec_ok)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long bars[3 * H_STAGES + 1];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ volatile int abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int64_t n0 = (int64_t)blockIdx.x * BM;
+    const int64_t m0 = (int64_t)blockIdx.y * BN;
+    const int64_t m_rows = (M - m0) < BN ? (M - m0) : BN;
+    const uint32_t n_mma = (uint32_t)((m_rows + 15) / 16 * 16);
+    const int n_half = (int)(n_mma / 2);
+    const int64_t kt0 = (int64_t)blockIdx.z * kt_split;
+    const int64_t kt_left = (D + BK - 1) / BK - kt0;
+    const int64_t ktiles = kt_left < kt_split ? (kt_left > 0 ? kt_left : 0) : kt_split;
+    const bool add_out = gridDim.z > 1;
+
+    // landed[s]: this CTA's two tiles of stage s have arrived; full[s] (used in the leader): both CTAs' tiles have;
+    // empty[s]: the MMAs that read stage s are done (both CTAs); accum: the accumulators are complete
+    const uint32_t landed0 = smem_u32(&bars[0]), full0 = smem_u32(&bars[H_STAGES]), empty0 = smem_u32(&bars[2 * H_STAGES]);
+    const uint32_t accum = smem_u32(&bars[3 * H_STAGES]);
+    if (tid == 0) {
+        for (int s = 0; s < H_STAGES; ++s) {
+            mbar_init(landed0 + 8 * s, 1);
+            mbar_init(full0 + 8 * s, 2);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(accum, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == H_EPI_WARPS) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                     "r"(H_TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync_all();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = tmem_base_slot;
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (warp < H_EPI_WARPS) {
+        // ---------------- epilogue: this CTA's 128 rows of the accumulator ----------------
+        bool ok = true;
+        if (ktiles > 0) ok = mbar_wait(accum, 0) && !abort_flag;
+        if (!ok) abort_flag = 1;
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int64_t row = n0 + warp * 32 + lane;
+        for (uint32_t c0 = 0; c0 < n_mma; c0 += 32) {
+            uint32_t v[32];
+            if (ok && ktiles > 0) {
+                tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + c0, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[e] = (ktiles > 0) ? 0x7FC00000u : 0u;   // NaN marks an aborted tile
+            }
+            if (row < N) {
+                float* dst = scores + row * ld_s + m0 + c0;
+                const bool vec = out_vec_ok && (int64_t)(c0 + 32) <= m_rows;
+                if (add_out) {
+                    if (vec) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + e),
+                                         "f"(__uint_as_float(v[e])), "f"(__uint_as_float(v[e + 1])),
+                                         "f"(__uint_as_float(v[e + 2])), "f"(__uint_as_float(v[e + 3]))
+                                         : "memory");
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if ((int64_t)(c0 + e) < m_rows) atomicAdd(dst + e, __uint_as_float(v[e]));
+                    }
+                } else if (vec) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4)
+                        *reinterpret_cast<uint4*>(dst + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if ((int64_t)(c0 + e) < m_rows) dst[e] = __uint_as_float(v[e]);
+                }
+            }
+        }
+    } else if (warp == H_EPI_WARPS + 1) {
+        // ---------------- TMA: bf16 tiles straight into the operand stages ----------------
+        // A tile arrives as H_BOXES boxes of H_BOX_ROWS rows, one box per lane.
+        const int32_t row_a = (int32_t)n0, row_b = (int32_t)(m0 + (int64_t)rank * n_half);
+        int64_t issued = 0;
+        bool ok = true;
+        for (int64_t kt = 0; kt < ktiles; ++kt) {
+            const int s = (int)(kt % H_STAGES);
+            const uint32_t round = (uint32_t)(kt / H_STAGES);
+            if (lane == 0) {
+                if (round > 0) ok = mbar_wait(empty0 + 8 * s, (round - 1) & 1) && !abort_flag;
+                if (ok) mbar_expect_tx(landed0 + 8 * s, H_STAGE_BYTES);
+            }
+            ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            if (lane < 2 * H_BOXES) {
+                const bool is_b = lane >= H_BOXES;
+                const int bx = is_b ? lane - H_BOXES : lane;
+                const uint32_t dst = smem_base + s * H_STAGE_BYTES + (is_b ? H_A_BYTES : 0) + bx * H_BOX_ROWS * (int)ROW_BYTES;
+                tma_load_2d(dst, is_b ? &map_test : &map_train, (int32_t)((kt0 + kt) * BK),
+                            (is_b ? row_b : row_a) + bx * H_BOX_ROWS, landed0 + 8 * s);
+            }
+            issued = kt + 1;
+        }
+        if (!ok) abort_flag = 1;
+        // no copy of this CTA may still be in flight when it leaves
+        if (lane == 0)
+            for (int64_t kt = issued > H_STAGES ? issued - H_STAGES : 0; kt < issued; ++kt)
+                if (!mbar_wait(landed0 + 8 * (int)(kt % H_STAGES), (uint32_t)(kt / H_STAGES) & 1)) abort_flag = 1;
+    } else if (warp == H_EPI_WARPS + 2) {
+        // ---------------- forward "landed" to the leader CTA ----------------
+        // An arrival on another CTA's barrier takes about a microsecond to return, so one thread forwarding
+        // stage after stage would set the pace of the whole kernel.  Lane s looks after stage s instead: the
+        // arrivals of several stages are in flight together; every lane polls once per turn of the common loop.
+        const uint32_t leader_full0 = map_to_cta(full0, 0);
+        int64_t kt = lane;
+        bool active = lane < H_STAGES;
+        uint32_t spins = 0;
+        while (__any_sync(0xFFFFFFFFu, active && kt < ktiles)) {
+            if (active && kt < ktiles) {
+                uint32_t done;
+                asm volatile(
+                    "{\n\t.reg .pred P;\n\t"
+                    "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+                    "selp.u32 %0, 1, 0, P;\n\t}"
+                    : "=r"(done)
+                    : "r"(landed0 + 8 * lane), "r"((uint32_t)(kt / H_STAGES) & 1)
+                    : "memory");
+                if (done) {
+                    mbar_arrive_cluster(leader_full0 + 8 * lane);
+                    kt += H_STAGES;
+                    spins = 0;
+                } else if (++spins > SPIN_LIMIT || abort_flag) {
+                    abort_flag = 1;
+                    active = false;
+                }
+            }
+        }
+    } else if (lane == 0 && rank == 0) {
+        // ---------------- MMA issuer (leader CTA only) ----------------
+        const uint32_t idesc = make_idesc(2 * BM, n_mma);
+        bool ok = true;
+        for (int64_t kt = 0; kt < ktiles && ok; ++kt) {
+            const int s = (int)(kt % H_STAGES);
+            ok = mbar_wait_cluster(full0 + 8 * s, (uint32_t)(kt / H_STAGES) & 1) && !abort_flag;
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a0 = smem_base + s * H_STAGE_BYTES, b0 = a0 + H_A_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < BK / 16; ++ks)
+                umma_bf16_pair(tmem_d, make_smem_desc(a0 + ks * 32), make_smem_desc(b0 + ks * 32), idesc,
+                               (kt > 0 || ks > 0) ? 1u : 0u);
+            umma_commit_pair(empty0 + 8 * s);
+        }
+        if (!ok) abort_flag = 1;
+        if (ok && ktiles > 0) umma_commit_pair(accum);
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == H_EPI_WARPS) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(H_TMEM_COLS) : "memory");
+    }
+}
+
 }  // namespace tc
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link libcuda)
@@ -380,18 +583,22 @@ static EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// rows x D fp32 matrix with row stride ld, read in boxes of 128 rows x 32 k-values (128 bytes, 128-byte swizzle);
-// elements outside the matrix are delivered as zeros
-static bool make_map(CUtensorMap* map, const float* base, int64_t rows, int64_t D, int64_t ld)
+// rows x D matrix with row stride ld, read in boxes of box_rows rows x 32 k-values: fp32 (128-byte rows, 128-byte
+// swizzle) or bf16 (64-byte rows, 64-byte swizzle: the operand layout itself); elements outside the matrix are
+// delivered as zeros
+static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t D, int64_t ld, bool bf16 = false,
+                     int box_rows = tc::BM)
 {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
+    const size_t esz = bf16 ? 2 : 4;
     const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)rows};
-    const cuuint64_t gstride[1] = {(cuuint64_t)ld * sizeof(float)};
-    const cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)tc::BM};
+    const cuuint64_t gstride[1] = {(cuuint64_t)ld * esz};
+    const cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows};
     const cuuint32_t estride[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), gdim, gstride, box, estride,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+    return enc(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base),
+               gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -400,6 +607,27 @@ bool score_tc_supported(const float* train, int64_t ld_train, const float* test,
 {
     return D > 0 && ((uintptr_t)train % 16 == 0) && ((uintptr_t)test % 16 == 0) && (ld_train % 4 == 0) &&
            (ld_test % 4 == 0) && encode_tiled_fn() != nullptr;
+}
+
+// Split of the contraction over blockIdx.z, for two reasons.  Accuracy: the tensor core truncates the fp32
+// accumulator after every MMA, a bias that grows with the number of accumulations, so one accumulator
+// never runs over more than 8,192 k-values once D exceeds 16,384 (the partial sums are then added in
+// round-to-nearest fp32).  Occupancy: with fewer tile pairs than SM pairs, k is split until the machine
+// is about full, in pieces of at least 256 k-values.
+static grass_status plan_splits(int64_t D, int64_t pairs, int64_t* splits_out, int64_t* kt_split_out)
+{
+    const int64_t ktiles = (D + tc::BK - 1) / tc::BK;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    int64_t splits = D > 16384 ? (D + 8191) / 8192 : 1;
+    if (pairs > 0 && pairs * 2 <= sms / 2) splits = std::max<int64_t>(splits, std::min<int64_t>(sms / 2 / pairs, D / 256));
+    if (const char* e = std::getenv("GRASS_SCORE_SPLITS")) splits = std::atoll(e);
+    splits = std::max<int64_t>(1, std::min<int64_t>(splits, std::min<int64_t>(ktiles, 65535)));
+    const int64_t kt_split = (ktiles + splits - 1) / splits;
+    *splits_out = (ktiles + kt_split - 1) / kt_split;
+    *kt_split_out = kt_split;
+    return GRASS_OK;
 }
 
 grass_status launch_score_tc(const float* train, int64_t N, int64_t ld_train, const float* test, int64_t M,
@@ -415,22 +643,8 @@ grass_status launch_score_tc(const float* train, int64_t N, int64_t ld_train, co
     if (cudaFuncSetAttribute(tc::grass_score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
         return GRASS_ERR_CUDA;
-    // Split of the contraction over blockIdx.z, for two reasons.  Accuracy: the tensor core truncates the fp32
-    // accumulator after every MMA, a bias that grows with the number of accumulations, so one accumulator
-    // never runs over more than 8,192 k-values once D exceeds 16,384 (the partial sums are then added in
-    // round-to-nearest fp32).  Occupancy: with fewer tile pairs than SM pairs, k is split until the machine
-    // is about full, in pieces of at least 256 k-values.
-    const int64_t ktiles = (D + tc::BK - 1) / tc::BK;
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
-    const int64_t pairs = gx / 2 * gy;
-    int64_t splits = D > 16384 ? (D + 8191) / 8192 : 1;
-    if (pairs > 0 && pairs * 2 <= sms / 2) splits = std::max<int64_t>(splits, std::min<int64_t>(sms / 2 / pairs, D / 256));
-    if (const char* e = std::getenv("GRASS_SCORE_SPLITS")) splits = std::atoll(e);
-    splits = std::max<int64_t>(1, std::min<int64_t>(splits, std::min<int64_t>(ktiles, 65535)));
-    const int64_t kt_split = (ktiles + splits - 1) / splits;
-    splits = (ktiles + kt_split - 1) / kt_split;
+    int64_t splits = 1, kt_split = 1;
+    if (plan_splits(D, gx / 2 * gy, &splits, &kt_split) != GRASS_OK) return GRASS_ERR_CUDA;
     if (splits > 1 &&
         cudaMemset2DAsync(scores, (size_t)ld_s * sizeof(float), 0, (size_t)M * sizeof(float), (size_t)N, st) != cudaSuccess)
         return GRASS_ERR_CUDA;
@@ -438,6 +652,39 @@ grass_status launch_score_tc(const float* train, int64_t N, int64_t ld_train, co
     const int out_vec_ok = ((uintptr_t)scores % 16 == 0) && (ld_s % 4 == 0);
     tc::grass_score_tc_kernel<<<grid, tc::THREADS, smem, st>>>(map_train, map_test, N, M, D, kt_split, scores, ld_s,
                                                                out_vec_ok);
+    return launch_status();
+}
+
+bool score_bf16_supported(const void* train, int64_t ld_train, const void* test, int64_t ld_test, int64_t D)
+{
+    return D > 0 && ((uintptr_t)train % 16 == 0) && ((uintptr_t)test % 16 == 0) && (ld_train % 8 == 0) &&
+           (ld_test % 8 == 0) && encode_tiled_fn() != nullptr;
+}
+
+grass_status launch_score_bf16(const void* train, int64_t N, int64_t ld_train, const void* test, int64_t M,
+                               int64_t ld_test, int64_t D, float* scores, int64_t ld_s, cudaStream_t st)
+{
+    const int64_t gx = ((N + tc::BM - 1) / tc::BM + 1) / 2 * 2;
+    const int64_t gy = (M + tc::BN - 1) / tc::BN;
+    if (gx > 0x7FFFFFFFLL || gy > 65535 || N > 0x7FFFFFFFLL || M > 0x7FFFFFFFLL || D > 0x7FFFFFFFLL)
+        return GRASS_ERR_UNSUPPORTED;
+    CUtensorMap map_train, map_test;
+    if (!make_map(&map_train, train, N, D, ld_train, true, tc::H_BOX_ROWS) ||
+        !make_map(&map_test, test, M, D, ld_test, true, tc::H_BOX_ROWS))
+        return GRASS_ERR_CUDA;
+    const size_t smem = (size_t)tc::H_STAGES * tc::H_STAGE_BYTES + 1024;
+    if (cudaFuncSetAttribute(tc::grass_score_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+        return GRASS_ERR_CUDA;
+    int64_t splits = 1, kt_split = 1;
+    if (plan_splits(D, gx / 2 * gy, &splits, &kt_split) != GRASS_OK) return GRASS_ERR_CUDA;
+    if (splits > 1 &&
+        cudaMemset2DAsync(scores, (size_t)ld_s * sizeof(float), 0, (size_t)M * sizeof(float), (size_t)N, st) != cudaSuccess)
+        return GRASS_ERR_CUDA;
+    dim3 grid((unsigned)gx, (unsigned)gy, (unsigned)splits);
+    const int out_vec_ok = ((uintptr_t)scores % 16 == 0) && (ld_s % 4 == 0);
+    tc::grass_score_bf16_kernel<<<grid, tc::H_THREADS, smem, st>>>(map_train, map_test, N, M, D, kt_split, scores, ld_s,
+                                                                   out_vec_ok);
     return launch_status();
 }
 
