@@ -374,7 +374,10 @@ constexpr int H_STAGES = GRASS_H_STAGES;
 constexpr int H_A_BYTES = BM * BK * 2;                   // this CTA's 128 train rows x 32 k-values of bf16: 8 KB
 constexpr int H_B_BYTES = BNH * BK * 2;                  // this CTA's half of the test rows: 8 KB
 constexpr int H_STAGE_BYTES = H_A_BYTES + H_B_BYTES;
-constexpr int H_BOX_ROWS = 32;                           // rows per TMA box
+#ifndef GRASS_H_BOX_ROWS
+#define GRASS_H_BOX_ROWS 128
+#endif
+constexpr int H_BOX_ROWS = GRASS_H_BOX_ROWS;                           // rows per TMA box
 constexpr int H_BOXES = BM / H_BOX_ROWS;                 // boxes per operand tile
 constexpr int H_EPI_WARPS = 4;
 constexpr int H_THREADS = (H_EPI_WARPS + 3) * 32;        // + MMA / tensor-memory warp, TMA warp, forwarding warp
