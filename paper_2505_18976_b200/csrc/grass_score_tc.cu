@@ -363,16 +363,18 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
 
 // ---------------------------------------------------------------------------------------------------------
 // The same contraction for vectors already stored as bf16 (a cache of compressed gradients at half the size):
-// no split is needed, so there are no producer warps at all.  TMA writes the bf16 tiles (128 rows x 32 k-values,
-// 64-byte swizzle) straight into the K-major operand layout the tensor core reads; per CTA one warp issues the
+// no split is needed, so there are no producer warps at all.  TMA writes the bf16 tiles (128 rows x 64 k-values,
+// 128-byte rows, 128-byte swizzle) straight into the K-major operand layout the tensor core reads; per CTA one warp issues the
 // loads, one forwards "my tiles have landed" to the leader CTA's barriers, one thread of the leader issues the
 // MMAs (one product per 16 k-values), four warps drain the accumulator.
 #ifndef GRASS_H_STAGES
-#define GRASS_H_STAGES 8
+#define GRASS_H_STAGES 6
 #endif
 constexpr int H_STAGES = GRASS_H_STAGES;
-constexpr int H_A_BYTES = BM * BK * 2;                   // this CTA's 128 train rows x 32 k-values of bf16: 8 KB
-constexpr int H_B_BYTES = BNH * BK * 2;                  // this CTA's half of the test rows: 8 KB
+constexpr int H_BK = 64;                                 // k-values per stage: 128-byte rows, 128-byte swizzle
+constexpr int H_ROW_BYTES = H_BK * 2;
+constexpr int H_A_BYTES = BM * H_ROW_BYTES;              // this CTA's 128 train rows x 64 k-values of bf16: 16 KB
+constexpr int H_B_BYTES = BNH * H_ROW_BYTES;             // this CTA's half of the test rows: 16 KB
 constexpr int H_STAGE_BYTES = H_A_BYTES + H_B_BYTES;
 #ifndef GRASS_H_BOX_ROWS
 #define GRASS_H_BOX_ROWS 128
@@ -382,9 +384,19 @@ constexpr int H_BOXES = BM / H_BOX_ROWS;                 // boxes per operand ti
 constexpr int H_EPI_WARPS = 4;
 constexpr int H_THREADS = (H_EPI_WARPS + 3) * 32;        // + MMA / tensor-memory warp, TMA warp, forwarding warp
 constexpr uint32_t H_TMEM_COLS = 256;                    // one fp32 accumulator of BN columns
-static_assert(H_STAGE_BYTES % 1024 == 0 && H_A_BYTES % 512 == 0, "operand tiles stay 512-byte aligned");
-static_assert(H_STAGES <= 32 && 2 * H_BOXES <= 32 && BM == BNH && (H_BOX_ROWS * ROW_BYTES) % 512 == 0,
+static_assert(H_STAGE_BYTES % 1024 == 0 && H_A_BYTES % 1024 == 0, "operand tiles stay 1024-byte aligned");
+static_assert(H_STAGES <= 32 && 2 * H_BOXES <= 32 && BM == BNH && (H_BOX_ROWS * H_ROW_BYTES) % 1024 == 0,
               "one stage and one box per lane");
+static_assert(H_STAGES * H_STAGE_BYTES <= 200 * 1024, "shared memory");
+
+// shared-memory matrix descriptor for K-major tiles with 128-byte rows and the 128-byte swizzle (8-row groups
+// 1,024 bytes apart; 16-byte chunk c of row r stored at chunk c ^ (r & 7)); a descriptor that starts 32 * i bytes
+// into the tile addresses k-values 16 i .. 16 i + 15
+__device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t addr)
+{
+    return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(H_THREADS, 1)
 grass_score_bf16_kernel(const __grid_constant__ CUtensorMap map_train, const __grid_constant__ CUtensorMap map_test,
@@ -404,7 +416,7 @@ grass_score_bf16_kernel(const __grid_constant__ CUtensorMap map_train, const __g
     const uint32_t n_mma = (uint32_t)((m_rows + 15) / 16 * 16);
     const int n_half = (int)(n_mma / 2);
     const int64_t kt0 = (int64_t)blockIdx.z * kt_split;
-    const int64_t kt_left = (D + BK - 1) / BK - kt0;
+    const int64_t kt_left = (D + H_BK - 1) / H_BK - kt0;
     const int64_t ktiles = kt_left < kt_split ? (kt_left > 0 ? kt_left : 0) : kt_split;
     const bool add_out = gridDim.z > 1;
 
@@ -497,8 +509,8 @@ grass_score_bf16_kernel(const __grid_constant__ CUtensorMap map_train, const __g
             if (lane < 2 * H_BOXES) {
                 const bool is_b = lane >= H_BOXES;
                 const int bx = is_b ? lane - H_BOXES : lane;
-                const uint32_t dst = smem_base + s * H_STAGE_BYTES + (is_b ? H_A_BYTES : 0) + bx * H_BOX_ROWS * (int)ROW_BYTES;
-                tma_load_2d(dst, is_b ? &map_test : &map_train, (int32_t)((kt0 + kt) * BK),
+                const uint32_t dst = smem_base + s * H_STAGE_BYTES + (is_b ? H_A_BYTES : 0) + bx * H_BOX_ROWS * H_ROW_BYTES;
+                tma_load_2d(dst, is_b ? &map_test : &map_train, (int32_t)((kt0 + kt) * H_BK),
                             (is_b ? row_b : row_a) + bx * H_BOX_ROWS, landed0 + 8 * s);
             }
             issued = kt + 1;
@@ -548,8 +560,8 @@ grass_score_bf16_kernel(const __grid_constant__ CUtensorMap map_train, const __g
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t a0 = smem_base + s * H_STAGE_BYTES, b0 = a0 + H_A_BYTES;
 #pragma unroll
-            for (int ks = 0; ks < BK / 16; ++ks)
-                umma_bf16_pair(tmem_d, make_smem_desc(a0 + ks * 32), make_smem_desc(b0 + ks * 32), idesc,
+            for (int ks = 0; ks < H_BK / 16; ++ks)
+                umma_bf16_pair(tmem_d, make_smem_desc_sw128(a0 + ks * 32), make_smem_desc_sw128(b0 + ks * 32), idesc,
                                (kt > 0 || ks > 0) ? 1u : 0u);
             umma_commit_pair(empty0 + 8 * s);
         }
@@ -586,8 +598,8 @@ static EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// rows x D matrix with row stride ld, read in boxes of box_rows rows x 32 k-values: fp32 (128-byte rows, 128-byte
-// swizzle) or bf16 (64-byte rows, 64-byte swizzle: the operand layout itself); elements outside the matrix are
+// rows x D matrix with row stride ld, read in boxes of box_rows rows x 128 bytes with the 128-byte swizzle: 32 fp32
+// k-values, or 64 bf16 k-values (then the box is an operand tile as it stands); elements outside the matrix are
 // delivered as zeros
 static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t D, int64_t ld, bool bf16 = false,
                      int box_rows = tc::BM)
@@ -597,11 +609,11 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t D
     const size_t esz = bf16 ? 2 : 4;
     const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)rows};
     const cuuint64_t gstride[1] = {(cuuint64_t)ld * esz};
-    const cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows};
+    const cuuint32_t box[2] = {(cuuint32_t)(bf16 ? tc::H_BK : tc::BK), (cuuint32_t)box_rows};
     const cuuint32_t estride[2] = {1, 1};
     return enc(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base),
                gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -617,9 +629,9 @@ bool score_tc_supported(const float* train, int64_t ld_train, const float* test,
 // never runs over more than 8,192 k-values once D exceeds 16,384 (the partial sums are then added in
 // round-to-nearest fp32).  Occupancy: with fewer tile pairs than SM pairs, k is split until the machine
 // is about full, in pieces of at least 256 k-values.
-static grass_status plan_splits(int64_t D, int64_t pairs, int64_t* splits_out, int64_t* kt_split_out)
+static grass_status plan_splits(int64_t D, int64_t pairs, int bk, int64_t* splits_out, int64_t* kt_split_out)
 {
-    const int64_t ktiles = (D + tc::BK - 1) / tc::BK;
+    const int64_t ktiles = (D + bk - 1) / bk;
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
@@ -647,7 +659,7 @@ grass_status launch_score_tc(const float* train, int64_t N, int64_t ld_train, co
         cudaSuccess)
         return GRASS_ERR_CUDA;
     int64_t splits = 1, kt_split = 1;
-    if (plan_splits(D, gx / 2 * gy, &splits, &kt_split) != GRASS_OK) return GRASS_ERR_CUDA;
+    if (plan_splits(D, gx / 2 * gy, tc::BK, &splits, &kt_split) != GRASS_OK) return GRASS_ERR_CUDA;
     if (splits > 1 &&
         cudaMemset2DAsync(scores, (size_t)ld_s * sizeof(float), 0, (size_t)M * sizeof(float), (size_t)N, st) != cudaSuccess)
         return GRASS_ERR_CUDA;
@@ -680,7 +692,7 @@ grass_status launch_score_bf16(const void* train, int64_t N, int64_t ld_train, c
         cudaSuccess)
         return GRASS_ERR_CUDA;
     int64_t splits = 1, kt_split = 1;
-    if (plan_splits(D, gx / 2 * gy, &splits, &kt_split) != GRASS_OK) return GRASS_ERR_CUDA;
+    if (plan_splits(D, gx / 2 * gy, tc::H_BK, &splits, &kt_split) != GRASS_OK) return GRASS_ERR_CUDA;
     if (splits > 1 &&
         cudaMemset2DAsync(scores, (size_t)ld_s * sizeof(float), 0, (size_t)M * sizeof(float), (size_t)N, st) != cudaSuccess)
         return GRASS_ERR_CUDA;
