@@ -368,7 +368,7 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
 // loads, one forwards "my tiles have landed" to the leader CTA's barriers, one thread of the leader issues the
 // MMAs (one product per 16 k-values), four warps drain the accumulator.
 #ifndef GRASS_H_STAGES
-#define GRASS_H_STAGES 6
+#define GRASS_H_STAGES 7
 #endif
 constexpr int H_STAGES = GRASS_H_STAGES;
 constexpr int H_BK = 64;                                 // k-values per stage: 128-byte rows, 128-byte swizzle
@@ -387,7 +387,7 @@ constexpr uint32_t H_TMEM_COLS = 256;                    // one fp32 accumulator
 static_assert(H_STAGE_BYTES % 1024 == 0 && H_A_BYTES % 1024 == 0, "operand tiles stay 1024-byte aligned");
 static_assert(H_STAGES <= 32 && 2 * H_BOXES <= 32 && BM == BNH && (H_BOX_ROWS * H_ROW_BYTES) % 1024 == 0,
               "one stage and one box per lane");
-static_assert(H_STAGES * H_STAGE_BYTES <= 200 * 1024, "shared memory");
+static_assert(H_STAGES * H_STAGE_BYTES <= 224 * 1024, "shared memory");
 
 // shared-memory matrix descriptor for K-major tiles with 128-byte rows and the 128-byte swizzle (8-row groups
 // 1,024 bytes apart; 16-byte chunk c of row r stored at chunk c ^ (r & 7)); a descriptor that starts 32 * i bytes
