@@ -32,6 +32,8 @@ METRIC = "per-sample gradients compressed/sec"
 UNIT = "samples/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 L2_BYTES = 126 * 1024 * 1024
+L2_FLUSHED = ("L2 flushed between steps: 252 MB written, then 252 MB read so that no modified lines are left to be "
+              "written back inside the timed step")
 
 
 # ----------------------------------------------------------------------------- plumbing
@@ -128,11 +130,20 @@ def barrier(world: int):
 
 
 class L2Flush:
-    def __init__(self, device):
-        self.buf = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+    """Evicts the inputs from L2 between timed steps: writes a buffer of twice the L2 size, then reads another
+    one of the same size.  The write alone would leave L2 full of modified lines, and their write-back (as much
+    DRAM traffic as a small workload's own reads) would land inside the next timed step; after the read pass
+    L2 holds only unmodified lines.  `clean=False` is the write alone (reported beside the default)."""
 
-    def __call__(self):
-        self.buf.zero_()
+    def __init__(self, device):
+        self.w = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device=device)
+        self.r = torch.zeros(2 * L2_BYTES // 8, dtype=torch.int64, device=device)
+        self.sink = None
+
+    def __call__(self, clean=True):
+        self.w.zero_()
+        if clean:
+            self.sink = self.r.sum()
 
 
 # ----------------------------------------------------------------------------- workloads (GPU arm)
@@ -167,7 +178,7 @@ class GrassJob:
         self.kernels_per_step = 2 * self.nbatch     # memset + compress kernel per call (upper bound)
         self.dominant = "grass_compress_kernel"
         self.l2 = (f"{self.ncopies} resident batch(es) of {batch_bytes / 1e6:.0f} MB rotated; "
-                   + ("input >> L2" if self.ncopies == 1 else "L2 flushed between steps"))
+                   + ("input >> L2" if self.ncopies == 1 else L2_FLUSHED))
         self.need_flush = self.ncopies > 1
         self._i = 0
 
@@ -237,7 +248,7 @@ class FactJob:
         self.kernels_per_step = 2 + (1 if self.score else 0) + ((2 + 3 * nb + 4 * nb) if self.precondition else 0)
         self.dominant = "factgrass_kernel"
         self.need_flush = self.dense < 4 * L2_BYTES
-        self.l2 = "L2 flushed between steps" if self.need_flush else "inputs >> L2"
+        self.l2 = L2_FLUSHED if self.need_flush else "inputs >> L2"
         self.ev = []
 
     def step(self, ev=None):
@@ -336,7 +347,7 @@ def time_job(job, steps, warmup, world, device):
         dom_ms = sum(a.elapsed_time(b) for a, b in dom_events) / len(dom_events)
     else:
         dom_ms = job.dominant_ms(total_ms / steps)
-    warm_ms = None
+    warm_ms = dirty_ms = None
     if flush is not None:
         # the same steps back to back with the inputs left in L2 (reported beside the cold figure, never as `value`)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -346,7 +357,18 @@ def time_job(job, steps, warmup, world, device):
         e1.record()
         torch.cuda.synchronize()
         warm_ms = max_over_ranks(e0.elapsed_time(e1) / steps, world, device)
-    return ms_per_step, dom_ms, warm_ms
+        # and cold after the write pass alone: L2 full of modified lines that the step has to write back
+        pairs = []
+        for _ in range(steps):
+            flush(clean=False)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            job.step()
+            e1.record()
+            pairs.append((e0, e1))
+        torch.cuda.synchronize()
+        dirty_ms = max_over_ranks(sum(a.elapsed_time(b) for a, b in pairs) / steps, world, device)
+    return ms_per_step, dom_ms, warm_ms, dirty_ms
 
 
 # ----------------------------------------------------------------------------- end-to-end (host buffers)
@@ -669,6 +691,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true",
+                    help="default workload only: skip the per_config object (configs 1-4 timed in the same run)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--small", action="store_true", help="reduced case for profiler captures (not a bench value)")
     ap.add_argument("--compare", action="store_true",
@@ -711,26 +735,37 @@ def main():
             print(json.dumps(compare_compressors(args.config if args.config >= 3 else 5, device, G, W)))
         return
 
-    job = make_job(args.config, device, G, W, small=args.small, seq_len_aware=args.seq_len_aware,
-                   fp32_inputs=args.fp32_inputs, precondition=args.precondition)
+    peaks, peak_src = load_peaks()
+
+    def measure(cfg_id, steps, **kw):
+        """One configuration, device-resident inputs: (job, ms per step, clocks, roofline object, extra config keys)."""
+        job = make_job(cfg_id, device, G, W, **kw)
+        sampler = ClockSampler(local)
+        sampler.start()
+        ms_per_step, dom_ms, warm_ms, dirty_ms = time_job(job, steps, warmup, world, device)
+        clocks = sampler.stop()
+        achieved = job.alg_bytes_per_launch / (dom_ms * 1e-3) / 1e9
+        plain = not (kw.get("fp32_inputs") or kw.get("seq_len_aware") or kw.get("small"))
+        roofline = {"bound": "hbm", "kernel": job.dominant, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src,
+                    "algorithmic_bytes_per_launch": int(job.alg_bytes_per_launch),
+                    "dense_bytes_per_launch": int(job.dense_bytes_per_launch), "ms_per_launch": dom_ms,
+                    "fetch64_bytes_per_launch": int(job.fetch_bytes_per_launch),
+                    "fetch64_achieved": job.fetch_bytes_per_launch / (dom_ms * 1e-3) / 1e9,
+                    "fetch64_frac": job.fetch_bytes_per_launch / (dom_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "traffic": TRAFFIC.get(cfg_id) if plain else None}
+        extra = {}
+        if warm_ms is not None:
+            extra["ms_per_step_l2_warm"] = warm_ms     # `ms_per_step` is the cold figure (L2 flushed before each step)
+            extra["ms_per_step_l2_modified"] = dirty_ms  # cold after the write pass alone (L2 full of modified lines)
+        return job, ms_per_step, clocks, roofline, extra
+
+    job, ms_per_step, clocks, roofline, extra = measure(args.config, args.steps, small=args.small,
+                                                        seq_len_aware=args.seq_len_aware, fp32_inputs=args.fp32_inputs,
+                                                        precondition=args.precondition)
     if args.fp32_inputs or args.precondition:
         args.no_e2e = True      # the host-buffer leg covers the default path only
-    sampler = ClockSampler(local)
-    sampler.start()
-    ms_per_step, dom_ms, warm_ms = time_job(job, args.steps, warmup, world, device)
-    clocks = sampler.stop()
     value = world * job.samples_per_step / (ms_per_step * 1e-3)
-
-    peaks, peak_src = load_peaks()
-    achieved = job.alg_bytes_per_launch / (dom_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": job.dominant, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src,
-                "algorithmic_bytes_per_launch": int(job.alg_bytes_per_launch),
-                "dense_bytes_per_launch": int(job.dense_bytes_per_launch), "ms_per_launch": dom_ms,
-                "fetch64_bytes_per_launch": int(job.fetch_bytes_per_launch),
-                "fetch64_achieved": job.fetch_bytes_per_launch / (dom_ms * 1e-3) / 1e9,
-                "fetch64_frac": job.fetch_bytes_per_launch / (dom_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                "traffic": None if (args.fp32_inputs or args.seq_len_aware or args.small) else TRAFFIC.get(args.config)}
 
     e2e = None
     if not args.no_e2e:
@@ -739,19 +774,47 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu = cpu_baseline(args.config, W)
 
+    # The default run also times the other four configurations (device-resident inputs, same cold-L2 protocol,
+    # fewer steps), so that one line carries all five; `value` stays the default workload's.
+    per_config = None
+    default_run = (args.config == 5 and not (args.small or args.fp32_inputs or args.precondition or args.seq_len_aware
+                                             or args.no_per_config))
+    if default_run:
+        main_desc = job.desc()
+        kernels_main = job.kernels_per_step * args.steps
+        del job
+        torch.cuda.empty_cache()
+        per_config = {}
+        for cid in (1, 2, 3, 4):
+            steps_c = max(3, min(args.steps, 20))
+            j, ms_c, clocks_c, roof_c, extra_c = measure(cid, steps_c)
+            d = j.desc()
+            d.update(extra_c)
+            v = world * j.samples_per_step / (ms_c * 1e-3)
+            per_config[f"c{cid}"] = {"value": v, "unit": UNIT, "ms_per_step": ms_c, "steps": steps_c,
+                                     "tokens_per_s": (v * j.cfg.T if cid >= 3 else None), "config": d,
+                                     "roofline": roof_c, "clocks": clocks_c,
+                                     "gpu_launches": j.kernels_per_step * steps_c}
+            del j
+            torch.cuda.empty_cache()
+    else:
+        main_desc = job.desc()
+        kernels_main = job.kernels_per_step * args.steps
+
     if rank == 0:
-        cfgd = job.desc()
+        cfgd = main_desc
         cfgd["replicas"] = world
-        if warm_ms is not None:
-            cfgd["ms_per_step_l2_warm"] = warm_ms      # `ms_per_step` is the cold figure (L2 flushed before each step)
+        cfgd.update(extra)
         if args.small:
             cfgd["small"] = True
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
                 "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16" if (args.config >= 3 and not args.fp32_inputs) else "f32", "data": "synthetic", "config": cfgd,
-                "tokens_per_s": (value * job.cfg.T if args.config >= 3 else None),
-                "clocks": clocks, "e2e": e2e, "gpu_launches": job.kernels_per_step * args.steps,
+                "tokens_per_s": (value * W.CONFIGS[args.config].T if args.config >= 3 else None),
+                "clocks": clocks, "e2e": e2e, "gpu_launches": kernels_main,
                 "roofline": roofline, "cpu_baseline": cpu}
+        if per_config is not None:
+            line["per_config"] = per_config
         print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist

@@ -12,7 +12,9 @@
  *
  * Conventions (all calls):
  *   - Pointers are DEVICE pointers unless the parameter is marked "host".  The caller owns every
- *     buffer; the library allocates nothing and keeps no state between calls.
+ *     buffer; the library allocates nothing and keeps no state between calls (the only exception is the
+ *     table of launch-shape overrides behind grass_set_tuning, a test hook that is empty unless set).
+ *     The library never reads the process environment.
  *   - The gathered inputs (g of grass_compress / grass_mask, A and G of the factgrass / factmask calls) may
  *     also be page-locked host memory that the device can address (cudaHostAlloc, cudaHostRegister): the
  *     kernels then read the masked elements in place across the bus, 64 bytes per touched piece, which for a
@@ -119,6 +121,10 @@ typedef struct {
  *              aligned, owned by the caller, in use until the work enqueued by this call has finished.
  *   out        B x ld_out fp32; each layer's [out_offset, out_offset + k) range is overwritten,
  *              ranges of different layers must not overlap.
+ * A layer whose kin or kout is 0 contributes a zeroed output range and is otherwise skipped.
+ * With L > 1 the descriptor table is copied from host memory owned by the call, so grouped calls
+ * (this one, the _varlen, factmask and _static variants) must not be recorded into a CUDA stream capture;
+ * a single layer (L == 1) travels as a kernel argument and has no such copy.
  */
 grass_status factgrass_compress_grouped(const factgrass_layer* layers /*host*/, int32_t L, grass_dtype dt,
                                         int32_t B, int32_t T, float* out, int64_t ld_out,
@@ -209,6 +215,9 @@ grass_status factgrass_compress_grouped_static(const factgrass_layer* layers /*h
  *   8,192 so that the relative accuracy does not degrade with D.  Whenever the contraction is split (long D,
  *   or few output tiles) the partial sums meet in the output, which the call first zeroes on the stream.
  * These are raw inner products of compressed gradients; preconditioning is the caller's.
+ * The call has no dev_status argument: should one of the kernel's bounded waits ever expire, the output tile
+ * of that thread block is filled with NaN (so the failure cannot pass for a score), its tensor memory is
+ * released and the kernel returns.  grass_score_bf16 follows the same convention.
  */
 grass_status grass_score(const float* train, int64_t N, int64_t ld_train, const float* test, int64_t M,
                          int64_t ld_test, int64_t D, float* scores, int64_t ld_s, void* stream);
@@ -276,6 +285,33 @@ grass_status grass_validate_mask(const uint32_t* idx, int64_t kprime, int64_t p,
 grass_status grass_random_mask_host(int64_t p, int64_t kprime, uint64_t seed, uint32_t* idx_host /*host*/);
 
 const char* grass_status_string(grass_status st);
+
+/*
+ * Launch-shape overrides (a test and measurement hook; the paper has no counterpart).  Every call above chooses
+ * its launch shape from the problem size.  The parity tests compare several shapes of the same kernel and the
+ * benchmark sweeps them, so each choice can be forced here.  value < 0 (GRASS_TUNE_AUTO) restores the automatic
+ * choice.  The table is process-wide and read at launch time; it is not meant to be changed while other threads
+ * are inside library calls.  Unknown keys return GRASS_ERR_INVALID_ARG.
+ */
+typedef enum {
+    GRASS_TUNE_COMPRESS_SAMPLES = 0,   /* grass_compress: samples per thread block (1, 2, 4, 8) */
+    GRASS_TUNE_COMPRESS_JSPLIT = 1,    /* grass_compress: thread blocks that share one sample's masked positions */
+    GRASS_TUNE_COMPRESS_CLUSTER = 2,   /* grass_compress: 0 = reduce position splits with global reductions */
+    GRASS_TUNE_COMPRESS_DENSE = 3,     /* grass_compress: 0 = no vector-load path for identity masks */
+    GRASS_TUNE_FACTGRASS_TILE = 4,     /* factgrass: block tile 64 or 128 */
+    GRASS_TUNE_FACTGRASS_CHUNK = 5,    /* factgrass: tokens per thread block */
+    GRASS_TUNE_FACTGRASS_CARVEOUT = 6, /* factgrass: shared-memory carve-out in percent */
+    GRASS_TUNE_SCORE_FFMA = 7,         /* grass_score: 1 = plain FMA kernel instead of the tensor-core one */
+    GRASS_TUNE_SCORE_SPLITS = 8,       /* grass_score, grass_score_bf16: splits of the contraction */
+    GRASS_TUNE_SPLIT_PRODUCTS = 9,     /* fp32 contractions: partial products per fp32 product (3, 4 or 6) */
+    GRASS_TUNE_FACTGRASS_PATH = 10,    /* factgrass: 0 = streaming kernel, 1 = cluster kernel (see factgrass.cu) */
+    GRASS_TUNE_FACTGRASS_STAGING = 11, /* factgrass cluster kernel: 0 = element gathers, 1 = whole token rows staged by TMA */
+    GRASS_TUNE_COMPRESS_LOADS = 12,    /* grass_compress gather path: loads in flight per thread (4, 8, 16) */
+    GRASS_TUNE_COMPRESS_THREADS = 13,  /* grass_compress gather path: threads per block (256, 512) */
+    GRASS_TUNE_COUNT = 14
+} grass_tuning_key;
+#define GRASS_TUNE_AUTO (-1)
+grass_status grass_set_tuning(grass_tuning_key key, int64_t value);
 
 #ifdef __cplusplus
 }

@@ -28,7 +28,13 @@ EXPORTS = ("grass_compress", "factgrass_compress", "factgrass_compress_grouped",
            "grass_fim", "grass_fim_factor", "grass_fim_apply", "grass_mask", "factmask_compress",
            "factmask_compress_grouped",
            "factgrass_grouped_workspace_bytes", "factgrass_compress_grouped_static", "grass_score", "grass_sjlt_table", "grass_validate_mask",
-           "grass_random_mask_host", "grass_status_string", "grass_to_bf16", "grass_score_bf16")
+           "grass_random_mask_host", "grass_status_string", "grass_to_bf16", "grass_score_bf16", "grass_set_tuning")
+
+# grass_tuning_key in include/grass.h
+TUNE = {"compress_samples": 0, "compress_jsplit": 1, "compress_cluster": 2, "compress_dense": 3,
+        "factgrass_tile": 4, "factgrass_chunk": 5, "factgrass_carveout": 6, "score_ffma": 7, "score_splits": 8,
+        "split_products": 9, "factgrass_path": 10, "factgrass_staging": 11, "compress_loads": 12,
+        "compress_threads": 13}
 
 
 class GrassError(RuntimeError):
@@ -104,6 +110,8 @@ def lib() -> ctypes.CDLL:
         L.grass_validate_mask.argtypes = [vp, i64, i64, vp]
         L.grass_random_mask_host.restype = st
         L.grass_random_mask_host.argtypes = [i64, i64, ctypes.c_uint64, vp]
+        L.grass_set_tuning.restype = st
+        L.grass_set_tuning.argtypes = [ctypes.c_int, i64]
         L.grass_status_string.restype = ctypes.c_char_p
         L.grass_status_string.argtypes = [st]
         _lib = L
@@ -149,6 +157,37 @@ def _need_device_readable(*ts) -> None:
             raise ValueError("device or pinned host tensors required (the library has no CPU path)")
 
 
+def _need_mask(*ms) -> None:
+    """Index lists are read as uint32: a 4-byte integer dtype, contiguous."""
+    for m in ms:
+        if m is not None and not isinstance(m, int):
+            if m.dtype not in (torch.int32, torch.uint32) or not m.is_contiguous() or m.dim() != 1:
+                raise TypeError("mask index lists must be contiguous 1-D int32/uint32 tensors")
+
+
+def grass_set_tuning(name: str, value: Optional[int]) -> None:
+    """Force one launch-shape choice of the library (a test and measurement hook); None restores automatic."""
+    _check(lib().grass_set_tuning(TUNE[name], -1 if value is None else int(value)), "grass_set_tuning")
+
+
+class tuning:
+    """Context manager: ``with tuning(factgrass_tile=128): ...`` forces the given choices and restores
+    automatic ones on exit."""
+
+    def __init__(self, **kw):
+        self.kw = kw
+
+    def __enter__(self):
+        for k, v in self.kw.items():
+            grass_set_tuning(k, v)
+        return self
+
+    def __exit__(self, *exc):
+        for k in self.kw:
+            grass_set_tuning(k, None)
+        return False
+
+
 def _compute_device(t: torch.Tensor) -> torch.device:
     return t.device if t.is_cuda else torch.device("cuda", torch.cuda.current_device())
 
@@ -161,6 +200,7 @@ def grass_compress(g: torch.Tensor, idx: Optional[torch.Tensor], k: int, s: int,
     g may be a pinned host tensor: the kernel then reads the masked elements in place, across the bus."""
     _need_device_readable(g)
     _need_cuda(idx, out, dev_status)
+    _need_mask(idx)
     assert g.dim() == 2 and g.stride(1) == 1
     n, ld = g.shape[0], g.stride(0) if g.shape[0] > 1 else g.shape[1]
     p = g.shape[1] if p is None else p
@@ -181,6 +221,7 @@ def factgrass_compress(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, 
     """One linear layer: out[b] = SJLT(vec(sum_t A[b,t,mask_in] (x) G[b,t,mask_out]))."""
     _need_device_readable(A, G)
     _need_cuda(mask_in, mask_out, out, dev_status)
+    _need_mask(mask_in, mask_out)
     assert A.is_contiguous() and G.is_contiguous() and A.dim() == 3 and G.dim() == 3
     B, T, d_in = A.shape
     d_out = G.shape[2]
@@ -213,7 +254,8 @@ def factgrass_compress_varlen(A: torch.Tensor, G: torch.Tensor, mask_in: torch.T
     int32 CUDA tensors; None = b * T_max / T_max)."""
     _need_device_readable(A, G)
     _need_cuda(mask_in, mask_out, out, dev_status)
-    assert A.is_contiguous() and G.is_contiguous()
+    _need_mask(mask_in, mask_out)
+    assert A.is_contiguous() and G.is_contiguous() and A.dtype == G.dtype
     _check_token_arrays(tok_begin, tok_count, B)
     d_in, d_out = A.shape[-1], G.shape[-1]
     if tok_begin is None:
@@ -241,6 +283,18 @@ class GroupedLayers:
         for i, l in enumerate(layers):
             _need_device_readable(l["A"], l["G"])
             _need_cuda(l["mask_in"], l["mask_out"])
+            _need_mask(l["mask_in"], l["mask_out"])
+            A0, Al, Gl = layers[0]["A"], l["A"], l["G"]
+            # every layer shares the token layout and dtype of the first; the kernels index with these
+            if not (Al.is_contiguous() and Gl.is_contiguous()):
+                raise ValueError(f"layer {i}: A and G must be contiguous")
+            if Al.dim() != A0.dim() or Gl.dim() != A0.dim() or Al.shape[:-1] != A0.shape[:-1] or \
+                    Gl.shape[:-1] != A0.shape[:-1]:
+                raise ValueError(f"layer {i}: A and G must share the leading (sample, token) shape of layer 0")
+            if Al.dtype != A0.dtype or Gl.dtype != A0.dtype:
+                raise TypeError(f"layer {i}: A and G must have the dtype of layer 0")
+            if l["out_offset"] < 0:
+                raise ValueError(f"layer {i}: negative out_offset")
             e = self.array[i]
             e.A, e.G = l["A"].data_ptr(), l["G"].data_ptr()
             e.mask_in, e.mask_out = l["mask_in"].data_ptr(), l["mask_out"].data_ptr()
@@ -354,6 +408,7 @@ def grass_mask(g: torch.Tensor, idx: torch.Tensor, out: Optional[torch.Tensor] =
     """Stand-alone Mask: out[i, j] = g[i, idx[j]] as fp32.  g may be a pinned host tensor (read in place)."""
     _need_device_readable(g)
     _need_cuda(idx, out, dev_status)
+    _need_mask(idx)
     assert g.dim() == 2 and g.stride(1) == 1
     n, ld = g.shape[0], g.stride(0) if g.shape[0] > 1 else g.shape[1]
     p = g.shape[1] if p is None else p
@@ -370,7 +425,9 @@ def factmask_compress(A: torch.Tensor, G: torch.Tensor, mask_in: torch.Tensor, m
     """Factorised Mask of one linear layer: out[b, a*kout + c] = sum_t A[b,t,mask_in[a]] G[b,t,mask_out[c]]."""
     _need_device_readable(A, G)
     _need_cuda(mask_in, mask_out, out, dev_status)
+    _need_mask(mask_in, mask_out)
     assert A.is_contiguous() and G.is_contiguous() and A.dim() == 3 and G.dim() == 3 and A.dtype == G.dtype
+    assert G.shape[:2] == A.shape[:2]
     B, T, d_in = A.shape
     d_out = G.shape[2]
     kin = d_in if mask_in is None else mask_in.numel()          # None = identity mask

@@ -71,7 +71,7 @@ __global__ void __launch_bounds__(kFgThreads)
 factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ LayerDesc single, int32_t B,
                  int32_t T, const int64_t* __restrict__ tok_begin, const int32_t* __restrict__ tok_count,
                  int32_t max_tiles, int32_t chunk_len, float* __restrict__ out, int64_t ld_out,
-                 uint32_t* dev_status)
+                 uint32_t* dev_status, int nprod)
 {
     using elem_t = typename in_elem<F32>::type;
     constexpr int NP = F32 ? 3 : 1;                       // bf16 pieces per operand
@@ -98,6 +98,9 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
     // HBM once and from L2 by the others
     const int chunk = blockIdx.x / max_tiles;
     const int tile = blockIdx.x % max_tiles;
+    // a layer with an empty factor mask has no block at all (its output range stays zero): leave before
+    // any division by its tile counts, any mask load or any allocation
+    if (L.tiles_m <= 0 || L.tiles_n <= 0) return;
     const int tm = tile % L.tiles_m, tn = tile / L.tiles_m;
     if (tn >= L.tiles_n) return;
     if (EPI == kEpiRaw && tn < tm) return;
@@ -219,14 +222,13 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
 #pragma unroll
             for (int ks = 0; ks < kTokTile / 16; ++ks) {
                 if constexpr (F32) {
-                    // (piece of A, piece of G): 0 = hi, 1 = mid, 2 = lo.  hi*hi goes to the first accumulator,
-                    // the five correction terms to the second (the tensor core truncates after every
-                    // accumulation, so the large sum sees as few of them as possible)
-                    const int pa[6] = {0, 2, 0, 1, 1, 0}, pg[6] = {0, 0, 2, 1, 0, 1};
+                    // hi*hi goes to the first accumulator, the correction terms to the second (the tensor core
+                    // truncates after every accumulation, so the large sum sees as few of them as possible)
 #pragma unroll
                     for (int q = 0; q < 6; ++q) {
-                        const uint64_t ad = tc::make_smem_desc(a0 + pa[q] * A_TILE + ks * 32);
-                        const uint64_t gd = tc::make_smem_desc(g0 + pg[q] * G_TILE + ks * 32);
+                        if (q >= nprod) break;
+                        const uint64_t ad = tc::make_smem_desc(a0 + tc::split_piece_a(q) * A_TILE + ks * 32);
+                        const uint64_t gd = tc::make_smem_desc(g0 + tc::split_piece_b(q) * G_TILE + ks * 32);
                         tc::umma_bf16(q == 0 ? tmem_d : tmem_d + TN, ad, gd, idesc, (it > 0 || ks > 0 || q > 1) ? 1u : 0u);
                     }
                 } else {
@@ -347,7 +349,9 @@ static grass_status fill_desc(LayerDesc& d, const factgrass_layer& l, int tile, 
         return GRASS_ERR_INVALID_ARG;
     if (l.out_offset < 0) return GRASS_ERR_INVALID_ARG;
     if ((l.kin > 0 && l.kout > 0 && T > 0) && (!l.A || !l.G)) return GRASS_ERR_INVALID_ARG;
-    if ((!l.mask_in && l.kin != l.d_in) || (!l.mask_out && l.kout != l.d_out)) return GRASS_ERR_INVALID_ARG;
+    // a NULL mask is the identity; an empty mask (k' = 0) needs no list either
+    if ((!l.mask_in && l.kin != l.d_in && l.kin != 0) || (!l.mask_out && l.kout != l.d_out && l.kout != 0))
+        return GRASS_ERR_INVALID_ARG;
     d.A = l.A;
     d.G = l.G;
     d.mask_in = l.mask_in;
@@ -365,12 +369,6 @@ static grass_status fill_desc(LayerDesc& d, const factgrass_layer& l, int tile, 
     d.use_smem_bins = (size_t)l.spec.k * sizeof(float) <= kMaxSmemBins;
     d.scale = 1.0f;
     return GRASS_OK;
-}
-
-static int fg_env_int(const char* name, int dflt)
-{
-    const char* v = std::getenv(name);
-    return v ? std::atoi(v) : dflt;
 }
 
 static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, grass_dtype dt, int32_t B, int32_t T,
@@ -396,8 +394,8 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
             return GRASS_ERR_INVALID_ARG;
     }
     // 64 x 64 block tiles; larger blocks are covered by several tiles whose shared rows come from L2.
-    // The 128 x 128 variant serves the projected FIM and comparison runs (FACTGRASS_TILE=128).
-    const int tile = fg_env_int("FACTGRASS_TILE", 64) == 128 && max_kk > 64 ? 128 : 64;
+    // The 128 x 128 variant serves the projected FIM and comparison runs (GRASS_TUNE_FACTGRASS_TILE = 128).
+    const int tile = tuning(GRASS_TUNE_FACTGRASS_TILE, 64) == 128 && max_kk > 64 ? 128 : 64;
 
     if (!workspace && L != 1) return GRASS_ERR_INVALID_ARG;
     if (workspace && (workspace_bytes < (size_t)L * sizeof(LayerDesc) || ((uintptr_t)workspace & 15)))
@@ -477,7 +475,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
             for (int kb : configs_kb)
                 if ((size_t)kb * 1024 >= (size_t)per_sm * cta_smem) { carve = kb * 100 / 228; break; }
         }
-        carve = fg_env_int("FACTGRASS_CARVEOUT", carve);
+        carve = (int)tuning(GRASS_TUNE_FACTGRASS_CARVEOUT, carve);
         if (cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, carve) != cudaSuccess)
             return GRASS_ERR_CUDA;
         // token chunks.  Every chunk pays a fixed projection epilogue (tile*tile hashes and a k-bin flush),
@@ -495,13 +493,15 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
         if (want < 1) want = 1;
         int chunk_len = (int)((T + want - 1) / want);
         chunk_len = (chunk_len + kTokTile - 1) / kTokTile * kTokTile;
-        chunk_len = fg_env_int("FACTGRASS_CHUNK", chunk_len);
+        chunk_len = (int)tuning(GRASS_TUNE_FACTGRASS_CHUNK, chunk_len);
         if (chunk_len < kTokTile) chunk_len = kTokTile;
         chunk_len = (chunk_len + kTokTile - 1) / kTokTile * kTokTile;
         const int nchunks = (T + chunk_len - 1) / chunk_len;
         dim3 grid((unsigned)(nchunks * max_tiles), (unsigned)B, (unsigned)L);
+        int nprod = (int)tuning(GRASS_TUNE_SPLIT_PRODUCTS, tc::kSplitProductsDefault);
+        if (nprod != 3 && nprod != 4) nprod = 6;
         kern<<<grid, kFgThreads, smem, st>>>(dev_descs, single, B, T, tok_begin, tok_count, max_tiles, chunk_len, out,
-                                             ld_out, dev_status);
+                                             ld_out, dev_status, nprod);
         return launch_status();
     };
     const size_t piece = (size_t)tile * tc::ROW_BYTES * 2;   // one bf16 piece of the A tile plus one of the G tile
@@ -575,8 +575,10 @@ grass_status launch_fim(const float* X, int64_t n, int64_t k, int64_t ld, float 
     const int64_t gx = nchunks * d.tiles_m * d.tiles_n;
     if (gx > 0x7FFFFFFFLL || chunk_len > 0x7FFFFFFFLL) return GRASS_ERR_UNSUPPORTED;
     dim3 grid((unsigned)gx, 1, 1);
+    int nprod = (int)tuning(GRASS_TUNE_SPLIT_PRODUCTS, tc::kSplitProductsDefault);
+    if (nprod != 3 && nprod != 4) nprod = 6;
     kern<<<grid, kFgThreads, smem, st>>>(nullptr, d, 1, (int32_t)n, nullptr, nullptr, d.tiles_m * d.tiles_n,
-                                         (int32_t)chunk_len, F, ld_f, nullptr);
+                                         (int32_t)chunk_len, F, ld_f, nullptr, nprod);
     return launch_status();
 }
 

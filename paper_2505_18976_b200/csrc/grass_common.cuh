@@ -49,60 +49,20 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t b)
     return __uint_as_float((uint32_t)b << 16);
 }
 
-#ifndef GRASS_LD_MODE
-#define GRASS_LD_MODE 6
-#endif
 // Gathered (scattered, read-once) loads of one element.  On B200 a plain load of an untouched 128-byte line makes
 // DRAM deliver the whole line; the L2::64B prefetch-size hint limits the fetch to the 64-byte half that holds the
 // element (nothing fetches less), which is what a sparse mask wants.  L1::no_allocate: the data are used once.
-// GRASS_LD_MODE selects other load forms for comparison builds.
 __device__ __forceinline__ uint32_t gather_u32(const uint32_t* p)
 {
-#if GRASS_LD_MODE == 0
-    return __ldg(p);
-#elif GRASS_LD_MODE == 1
-    return *p;
-#elif GRASS_LD_MODE == 2
-    return __ldcg(p);
-#elif GRASS_LD_MODE == 3
-    return __ldcs(p);
-#elif GRASS_LD_MODE == 4
-    uint32_t v;
-    asm volatile("ld.global.nc.L1::no_allocate.b32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-#elif GRASS_LD_MODE == 5
-    uint32_t v;
-    asm("ld.global.nc.L2::64B.b32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-#else
     uint32_t v;
     asm("ld.global.nc.L1::no_allocate.L2::64B.b32 %0, [%1];" : "=r"(v) : "l"(p));
     return v;
-#endif
 }
 __device__ __forceinline__ uint16_t gather_u16(const uint16_t* p)
 {
-#if GRASS_LD_MODE == 0
-    return __ldg(p);
-#elif GRASS_LD_MODE == 1
-    return *p;
-#elif GRASS_LD_MODE == 2
-    return __ldcg(p);
-#elif GRASS_LD_MODE == 3
-    return __ldcs(p);
-#elif GRASS_LD_MODE == 5
-    uint16_t v;
-    asm("ld.global.nc.L2::64B.b16 %0, [%1];" : "=h"(v) : "l"(p));
-    return v;
-#elif GRASS_LD_MODE == 6
     uint16_t v;
     asm("ld.global.nc.L1::no_allocate.L2::64B.b16 %0, [%1];" : "=h"(v) : "l"(p));
     return v;
-#else
-    uint16_t v;
-    asm volatile("ld.global.nc.L1::no_allocate.b16 %0, [%1];" : "=h"(v) : "l"(p));
-    return v;
-#endif
 }
 
 template <typename T> struct elem;
@@ -118,6 +78,9 @@ template <> struct elem<__nv_bfloat16> {
         return bf16_bits_to_float(gather_u16(reinterpret_cast<const uint16_t*>(p)));
     }
 };
+
+// launch-shape override set through grass_set_tuning, or `dflt` while the key is on automatic
+int64_t tuning(grass_tuning_key key, int64_t dflt);
 
 inline grass_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? GRASS_OK : GRASS_ERR_CUDA; }
 

@@ -14,7 +14,6 @@
 #include "grass_common.cuh"
 
 #include <cooperative_groups.h>
-#include <cstdlib>
 
 namespace cg = cooperative_groups;
 
@@ -288,12 +287,6 @@ struct CompressPlan {
     int cluster;    // the jsplit CTAs are one thread-block cluster (DSMEM reduction)
 };
 
-static int env_int(const char* name, int dflt)
-{
-    const char* v = std::getenv(name);
-    return v ? std::atoi(v) : dflt;
-}
-
 static CompressPlan plan_compress(int64_t n, int64_t kprime, uint32_t k, int sm_count, bool dense)
 {
     CompressPlan pl;
@@ -305,7 +298,7 @@ static CompressPlan plan_compress(int64_t n, int64_t kprime, uint32_t k, int sm_
     // gathered loads leave idle, so sharing it between samples buys nothing and costs occupancy.
     // Dense rows are the exception: every position is read, the hash is the larger cost, and two samples share it
     // where their bins still leave room for several CTAs per SM (four samples measured slower at k = 4,096).
-    int S = env_int("GRASS_COMPRESS_S", dense && bin_bytes * 2 <= 64 * 1024 ? 2 : 1);
+    int S = (int)tuning(GRASS_TUNE_COMPRESS_SAMPLES, dense && bin_bytes * 2 <= 64 * 1024 ? 2 : 1);
     if (S != 1 && S != 2 && S != 4 && S != 8) S = 1;
     while (S > 1 && pl.use_smem && bin_bytes * S > smem_cap) S >>= 1;
     if (!pl.use_smem) S = 1;
@@ -323,10 +316,10 @@ static CompressPlan plan_compress(int64_t n, int64_t kprime, uint32_t k, int sm_
         if (js > max_js) js = max_js;
         pl.cluster = 0;
     }
-    const int forced = env_int("GRASS_COMPRESS_JSPLIT", 0);
+    const int forced = (int)tuning(GRASS_TUNE_COMPRESS_JSPLIT, 0);
     if (forced > 0) {
         js = forced;
-        pl.cluster = forced <= 8 && env_int("GRASS_COMPRESS_CLUSTER", 1) != 0;
+        pl.cluster = forced <= 8 && tuning(GRASS_TUNE_COMPRESS_CLUSTER, 1) != 0;
     }
     if (js < 1) js = 1;
     if (js > 65535) js = 65535;
@@ -388,7 +381,7 @@ static grass_status dispatch_compress(const T* g, int64_t n, int64_t p, int64_t 
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
-    const bool dense = idx == nullptr && env_int("GRASS_COMPRESS_DENSE", 1) != 0 &&
+    const bool dense = idx == nullptr && tuning(GRASS_TUNE_COMPRESS_DENSE, 1) != 0 &&
                        (uintptr_t)g % (4 * sizeof(T)) == 0 && ld % 4 == 0;
     const CompressPlan pl = plan_compress(n, kprime, sp.k, sms, dense);
     if (!pl.cluster && (pl.jsplit > 1 || !pl.use_smem)) {

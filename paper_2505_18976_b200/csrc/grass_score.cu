@@ -3,7 +3,7 @@
 // grass_score_tc.cu); it loads with TMA and therefore wants 16-byte aligned bases and row strides.  This
 // file holds the entry point and the plain fp32 FMA kernel (128 x 128 output tile per CTA, 8 x 8 per
 // thread, 16-deep k tiles double-buffered through registers and shared memory) that takes every other
-// input (and D = 0); GRASS_SCORE_IMPL=ffma selects it for comparison runs.
+// input (and D = 0); the GRASS_TUNE_SCORE_FFMA override selects it for comparison runs.
 #include "grass_common.cuh"
 
 #include <cstdlib>
@@ -124,8 +124,7 @@ extern "C" grass_status grass_score(const float* train, int64_t N, int64_t ld_tr
     if (N < 0 || M < 0 || D < 0 || ld_train < D || ld_test < D || ld_s < M) return GRASS_ERR_INVALID_ARG;
     if (N == 0 || M == 0) return GRASS_OK;
     if (!scores || (D > 0 && (!train || !test))) return GRASS_ERR_INVALID_ARG;
-    const char* impl = std::getenv("GRASS_SCORE_IMPL");
-    if ((!impl || std::strcmp(impl, "ffma") != 0) && grass::score_tc_supported(train, ld_train, test, ld_test, D))
+    if (grass::tuning(GRASS_TUNE_SCORE_FFMA, 0) == 0 && grass::score_tc_supported(train, ld_train, test, ld_test, D))
         return grass::launch_score_tc(train, N, ld_train, test, M, ld_test, D, scores, ld_s, (cudaStream_t)stream);
     const int64_t gx = (N + grass::SC_BM - 1) / grass::SC_BM, gy = (M + grass::SC_BN - 1) / grass::SC_BN;
     if (gx > 0x7FFFFFFFLL || gy > 65535) return GRASS_ERR_UNSUPPORTED;

@@ -138,7 +138,7 @@ __device__ __forceinline__ void cluster_sync_all()
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __grid_constant__ CUtensorMap map_test,
                       int64_t N, int64_t M, int64_t D, int64_t kt_split, float* __restrict__ scores, int64_t ld_s,
-                      int out_vec_ok)
+                      int out_vec_ok, int nprod)
 {
     extern __shared__ __align__(1024) unsigned char smem[];
     __shared__ __align__(8) unsigned long long bars[2 * STAGES + 1 + 2 * RING];
@@ -331,16 +331,16 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t a0 = smem_base + s * STAGE_BYTES, b0 = a0 + 3 * A_SPLIT_BYTES;
-            // (piece of A, piece of B): 0 = hi, 1 = mid, 2 = lo.  hi*hi goes to the first accumulator, the
-            // five correction terms (2^-8 and 2^-16 of it) to the second: the tensor core truncates after
-            // every accumulation, so the large sum should see as few of them as possible
-            const int pa[6] = {0, 2, 0, 1, 1, 0}, pb[6] = {0, 0, 2, 1, 0, 1};
+            // hi*hi goes to the first accumulator, the correction terms (2^-8 and 2^-16 of it) to the second:
+            // the tensor core truncates after every accumulation, so the large sum should see as few of
+            // them as possible
 #pragma unroll
             for (int t = 0; t < 6; ++t) {
+                if (t >= nprod) break;
 #pragma unroll
                 for (int ks = 0; ks < BK / 16; ++ks) {
-                    const uint64_t ad = make_smem_desc(a0 + pa[t] * A_SPLIT_BYTES + ks * 32);   // 16 k values on
-                    const uint64_t bd = make_smem_desc(b0 + pb[t] * B_SPLIT_BYTES + ks * 32);
+                    const uint64_t ad = make_smem_desc(a0 + split_piece_a(t) * A_SPLIT_BYTES + ks * 32);   // 16 k values on
+                    const uint64_t bd = make_smem_desc(b0 + split_piece_b(t) * B_SPLIT_BYTES + ks * 32);
                     const uint32_t acc_on = (kt > 0 || ks > 0 || t > 1) ? 1u : 0u;
                     umma_bf16_pair(t == 0 ? tmem_d : tmem_d + BN, ad, bd, idesc, acc_on);
                 }
@@ -367,19 +367,13 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
 // 128-byte rows, 128-byte swizzle) straight into the K-major operand layout the tensor core reads; per CTA one warp issues the
 // loads, one forwards "my tiles have landed" to the leader CTA's barriers, one thread of the leader issues the
 // MMAs (one product per 16 k-values), four warps drain the accumulator.
-#ifndef GRASS_H_STAGES
-#define GRASS_H_STAGES 7
-#endif
-constexpr int H_STAGES = GRASS_H_STAGES;
+constexpr int H_STAGES = 7;
 constexpr int H_BK = 64;                                 // k-values per stage: 128-byte rows, 128-byte swizzle
 constexpr int H_ROW_BYTES = H_BK * 2;
 constexpr int H_A_BYTES = BM * H_ROW_BYTES;              // this CTA's 128 train rows x 64 k-values of bf16: 16 KB
 constexpr int H_B_BYTES = BNH * H_ROW_BYTES;             // this CTA's half of the test rows: 16 KB
 constexpr int H_STAGE_BYTES = H_A_BYTES + H_B_BYTES;
-#ifndef GRASS_H_BOX_ROWS
-#define GRASS_H_BOX_ROWS 128
-#endif
-constexpr int H_BOX_ROWS = GRASS_H_BOX_ROWS;                           // rows per TMA box
+constexpr int H_BOX_ROWS = 128;                          // rows per TMA box
 constexpr int H_BOXES = BM / H_BOX_ROWS;                 // boxes per operand tile
 constexpr int H_EPI_WARPS = 4;
 constexpr int H_THREADS = (H_EPI_WARPS + 3) * 32;        // + MMA / tensor-memory warp, TMA warp, forwarding warp
@@ -637,7 +631,7 @@ static grass_status plan_splits(int64_t D, int64_t pairs, int bk, int64_t* split
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
     int64_t splits = D > 16384 ? (D + 8191) / 8192 : 1;
     if (pairs > 0 && pairs * 2 <= sms / 2) splits = std::max<int64_t>(splits, std::min<int64_t>(sms / 2 / pairs, D / 256));
-    if (const char* e = std::getenv("GRASS_SCORE_SPLITS")) splits = std::atoll(e);
+    splits = tuning(GRASS_TUNE_SCORE_SPLITS, splits);
     splits = std::max<int64_t>(1, std::min<int64_t>(splits, std::min<int64_t>(ktiles, 65535)));
     const int64_t kt_split = (ktiles + splits - 1) / splits;
     *splits_out = (ktiles + kt_split - 1) / kt_split;
@@ -665,8 +659,10 @@ grass_status launch_score_tc(const float* train, int64_t N, int64_t ld_train, co
         return GRASS_ERR_CUDA;
     dim3 grid((unsigned)gx, (unsigned)gy, (unsigned)splits);
     const int out_vec_ok = ((uintptr_t)scores % 16 == 0) && (ld_s % 4 == 0);
+    int nprod = (int)tuning(GRASS_TUNE_SPLIT_PRODUCTS, tc::kSplitProductsDefault);
+    if (nprod != 3 && nprod != 4) nprod = 6;
     tc::grass_score_tc_kernel<<<grid, tc::THREADS, smem, st>>>(map_train, map_test, N, M, D, kt_split, scores, ld_s,
-                                                               out_vec_ok);
+                                                               out_vec_ok, nprod);
     return launch_status();
 }
 

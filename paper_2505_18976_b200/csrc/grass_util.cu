@@ -3,10 +3,22 @@
 #include "grass_common.cuh"
 
 #include <algorithm>
+#include <atomic>
 #include <unordered_set>
 #include <vector>
 
 namespace grass {
+
+// launch-shape overrides (grass_set_tuning); a negative entry means "automatic"
+static std::atomic<int64_t> g_tuning[GRASS_TUNE_COUNT];
+static std::atomic<bool> g_tuning_used{false};
+
+int64_t tuning(grass_tuning_key key, int64_t dflt)
+{
+    if (!g_tuning_used.load(std::memory_order_acquire)) return dflt;
+    const int64_t v = g_tuning[key].load(std::memory_order_relaxed);
+    return v < 0 ? dflt : v;
+}
 
 __global__ void sjlt_table_kernel(uint32_t k, uint32_t s, uint64_t seed, int64_t total, uint32_t* __restrict__ bucket,
                                   int8_t* __restrict__ sign)
@@ -104,6 +116,18 @@ extern "C" grass_status grass_random_mask_host(int64_t p, int64_t kprime, uint64
     }
     std::sort(picks.begin(), picks.end());
     std::copy(picks.begin(), picks.end(), idx_host);
+    return GRASS_OK;
+}
+
+extern "C" grass_status grass_set_tuning(grass_tuning_key key, int64_t value)
+{
+    if ((int)key < 0 || (int)key >= (int)GRASS_TUNE_COUNT) return GRASS_ERR_INVALID_ARG;
+    if (!grass::g_tuning_used.load(std::memory_order_acquire)) {
+        // first use: every key starts on automatic
+        for (int i = 0; i < (int)GRASS_TUNE_COUNT; ++i) grass::g_tuning[i].store(-1, std::memory_order_relaxed);
+        grass::g_tuning_used.store(true, std::memory_order_release);
+    }
+    grass::g_tuning[key].store(value < 0 ? -1 : value, std::memory_order_relaxed);
     return GRASS_OK;
 }
 

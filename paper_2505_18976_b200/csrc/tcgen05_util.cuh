@@ -111,26 +111,42 @@ __device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&v)
         : "memory");
 }
 
-// eight consecutive fp32 -> three 16-byte chunks of bf16 (hi, mid, lo), x = hi + mid + lo exactly
+// two fp32 -> one register of two bf16, round to nearest even, finite inputs stay finite (x0 in the low half)
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float x0, float x1)
+{
+    uint32_t r;
+    asm("cvt.rn.satfinite.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(x1), "f"(x0));
+    return r;
+}
+
+// eight consecutive fp32 -> three 16-byte chunks of bf16 (hi, mid, lo), x = hi + mid + lo exactly.
+// Every piece is the round-to-nearest bf16 of what the pieces before it left over: the two subtractions are
+// exact in fp32, the third piece is exact, and hi + mid alone is x rounded to 16-17 significant bits with an
+// error of either sign (at most 2^-18 |x|), so that sums of products built from two pieces carry no bias.
 __device__ __forceinline__ void split8(const float (&x)[8], uint4& hi, uint4& mid, uint4& lo)
 {
-    uint32_t h[8], m[8], l[8];
+    uint32_t h[4], m[4], l[4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const uint32_t xb = __float_as_uint(x[i]);
-        h[i] = xb & 0xFFFF0000u;
-        const float r1 = x[i] - __uint_as_float(h[i]);
-        m[i] = __float_as_uint(r1) & 0xFFFF0000u;
-        const float r2 = r1 - __uint_as_float(m[i]);
-        l[i] = __float_as_uint(r2);
+    for (int i = 0; i < 4; ++i) {
+        const float x0 = x[2 * i], x1 = x[2 * i + 1];
+        h[i] = pack_bf16x2_rn(x0, x1);
+        const float r0 = x0 - __uint_as_float(h[i] << 16), r1 = x1 - __uint_as_float(h[i] & 0xFFFF0000u);
+        m[i] = pack_bf16x2_rn(r0, r1);
+        const float s0 = r0 - __uint_as_float(m[i] << 16), s1 = r1 - __uint_as_float(m[i] & 0xFFFF0000u);
+        l[i] = pack_bf16x2_rn(s0, s1);
     }
-    hi = make_uint4(__byte_perm(h[0], h[1], 0x7632), __byte_perm(h[2], h[3], 0x7632), __byte_perm(h[4], h[5], 0x7632),
-                    __byte_perm(h[6], h[7], 0x7632));
-    mid = make_uint4(__byte_perm(m[0], m[1], 0x7632), __byte_perm(m[2], m[3], 0x7632), __byte_perm(m[4], m[5], 0x7632),
-                     __byte_perm(m[6], m[7], 0x7632));
-    lo = make_uint4(__byte_perm(l[0], l[1], 0x7632), __byte_perm(l[2], l[3], 0x7632), __byte_perm(l[4], l[5], 0x7632),
-                    __byte_perm(l[6], l[7], 0x7632));
+    hi = make_uint4(h[0], h[1], h[2], h[3]);
+    mid = make_uint4(m[0], m[1], m[2], m[3]);
+    lo = make_uint4(l[0], l[1], l[2], l[3]);
 }
+
+// Partial products of a split fp32 contraction, as (piece of the first operand, piece of the second), 0 = hi,
+// 1 = mid, 2 = lo, in the order of their weight: hi*hi; the two terms at 2^-8 of it; mid*mid (2^-16); the two
+// hi*lo terms (2^-16).  All six reproduce the fp32 product to 2^-23; the first four to about 2^-17 (unbiased);
+// the first three to about 2^-16.  The first goes to an accumulator of its own.
+__host__ __device__ constexpr int split_piece_a(int q) { return (q == 2 || q == 3) ? 1 : (q == 5 ? 2 : 0); }
+__host__ __device__ constexpr int split_piece_b(int q) { return (q == 1 || q == 3) ? 1 : (q == 4 ? 2 : 0); }
+constexpr int kSplitProductsDefault = 6;
 
 }  // namespace tc
 }  // namespace grass

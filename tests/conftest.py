@@ -31,3 +31,19 @@ def oracle_mod():
     import oracle
     oracle.build()
     return oracle
+
+
+@pytest.fixture
+def tune():
+    """tune(key=value, ...) forces launch-shape choices of the library through grass_set_tuning (None restores
+    the automatic choice); everything is back on automatic after the test."""
+    import paper_2505_18976_b200 as G
+    touched = set()
+
+    def set_(**kw):
+        for k, v in kw.items():
+            G.grass_set_tuning(k, v)
+            touched.add(k)
+    yield set_
+    for k in touched:
+        G.grass_set_tuning(k, None)

@@ -118,18 +118,18 @@ def test_grass_compress_identity_mask_and_stride(G, W, oracle_mod):
 
 
 @pytest.mark.parametrize("zero_prob", [0.0, 0.5, 0.9, 0.99, 0.999])
-def test_plain_sjlt_over_input_sparsity(G, W, oracle_mod, monkeypatch, zero_prob):
+def test_plain_sjlt_over_input_sparsity(G, W, oracle_mod, tune, zero_prob):
     """Identity mask on vector-aligned rows: rounds of loads with few non-zeros go through the per-warp queue, fuller
     ones are hashed in place; one and two samples per CTA, s = 1 and 2, fp32 and bf16, a ragged tail, an odd k,
     and a k whose bins do not fit in shared memory."""
     for S in (1, 2):
-        monkeypatch.setenv("GRASS_COMPRESS_S", str(S))
+        tune(compress_samples=S)
         _grass_case(G, W, oracle_mod, 9, 131_072, 131_072, 4_096, identity=True, zero_prob=zero_prob)
         _grass_case(G, W, oracle_mod, 5, 40_004, 40_004, 777, s=2, identity=True, zero_prob=zero_prob)
         _grass_case(G, W, oracle_mod, 4, 33_000, 33_000, 512, identity=True, zero_prob=zero_prob, dtype=torch.bfloat16)
-    monkeypatch.delenv("GRASS_COMPRESS_S")
+    tune(compress_samples=None)
     _grass_case(G, W, oracle_mod, 3, 70_000, 70_000, 60_000, identity=True, zero_prob=zero_prob)
-    monkeypatch.setenv("GRASS_COMPRESS_JSPLIT", "5")
+    tune(compress_jsplit=5)
     _grass_case(G, W, oracle_mod, 3, 50_000, 50_000, 300, identity=True, zero_prob=zero_prob)
 
 
@@ -158,11 +158,9 @@ def test_grass_compress_student_t(G, W, oracle_mod):
 
 @pytest.mark.parametrize("S,js,cluster", [(1, 1, 1), (2, 3, 0), (4, 7, 0), (8, 2, 1), (1, 2, 1), (1, 4, 1), (1, 8, 1),
                                           (2, 4, 1), (1, 8, 0), (1, 20, 1)])
-def test_grass_compress_launch_shapes(G, W, oracle_mod, monkeypatch, S, js, cluster):
+def test_grass_compress_launch_shapes(G, W, oracle_mod, tune, S, js, cluster):
     """Every plan (samples per CTA, position split, cluster or global-atomic reduction) gives the same answer."""
-    monkeypatch.setenv("GRASS_COMPRESS_S", str(S))
-    monkeypatch.setenv("GRASS_COMPRESS_JSPLIT", str(js))
-    monkeypatch.setenv("GRASS_COMPRESS_CLUSTER", str(cluster))
+    tune(compress_samples=S, compress_jsplit=js, compress_cluster=cluster)
     _grass_case(G, W, oracle_mod, 11, 40_000, 9_000, 1_000)
     _grass_case(G, W, oracle_mod, 5, 40_000, 9_000, 1_003, s=2)
 
@@ -286,25 +284,25 @@ def test_factgrass_fp32_inputs(G, W, oracle_mod, kw):
     assert rel < 1e-4
 
 
-def test_factgrass_fp32_tile128(G, W, oracle_mod, monkeypatch):
-    monkeypatch.setenv("FACTGRASS_TILE", "128")
+def test_factgrass_fp32_tile128(G, W, oracle_mod, tune):
+    tune(factgrass_tile=128)
     cfg = _fact_cfg(W, layers=(W.LinearLayer("l", 768, 3072),), kin=128, kout=128, k=4096, T=130, B=3)
     _fact_case(G, W, oracle_mod, cfg, dtype=torch.float32)
     _fact_case(G, W, oracle_mod, cfg)
 
 
 @pytest.mark.parametrize("chunk", [32, 64, 1 << 20])
-def test_factgrass_token_chunking(G, W, oracle_mod, monkeypatch, chunk):
+def test_factgrass_token_chunking(G, W, oracle_mod, tune, chunk):
     """Splitting the token sum over CTAs (linearity of SJLT) does not change the result."""
-    monkeypatch.setenv("FACTGRASS_CHUNK", str(chunk))
+    tune(factgrass_chunk=chunk)
     _fact_case(G, W, oracle_mod, _fact_cfg(W, T=250, kin=64, kout=64, k=512))
 
 
 @pytest.mark.parametrize("tile", [64, 128])
-def test_factgrass_seeded_shape_sweep(G, W, oracle_mod, monkeypatch, tile):
+def test_factgrass_seeded_shape_sweep(G, W, oracle_mod, tune, tile):
     """Seeded random shapes: layer widths, mask sizes around the 64 / 128 tile edges, token counts that end inside a
     32-token stage, output lengths on both sides of the block size, one or two draws, bf16 and fp32 factors."""
-    monkeypatch.setenv("FACTGRASS_TILE", str(tile))
+    tune(factgrass_tile=tile)
     rng = np.random.default_rng(1234 + tile)
     for case in range(10):
         d_in, d_out = int(rng.integers(8, 700)), int(rng.integers(8, 700))
@@ -429,6 +427,37 @@ def test_factgrass_grouped_mixed_layers(G, W, oracle_mod):
         check_close(host[:, o:o + k], ref, absum, TOL_BF16, T + 64, eps=EPS_TC, what=f"mixed off={o}")
 
 
+def test_factgrass_grouped_layer_with_an_empty_mask(G, W, oracle_mod):
+    """A layer whose input-factor mask is empty has no block: its output range must come back as zeros, the
+    other layers must be untouched by it, and no device fault may be flagged."""
+    B, T = 2, 70
+    specs = [(96, 160, 24, 40, 97), (200, 64, 0, 64, 128), (128, 128, 64, 0, 64), (768, 3072, 64, 64, 300)]
+    layers, refs, off = [], [], 0
+    for n, (d_in, d_out, kin, kout, k) in enumerate(specs):
+        cfg = _fact_cfg(W, layers=(W.LinearLayer("x", d_in, d_out),), B=B, T=T, kin=max(kin, 1), kout=max(kout, 1),
+                        k=k, data_seed=200 + n)
+        A, Gt = W.layer_io(cfg, 0, device="cuda")
+        mi = oracle_mod.random_mask(d_in, kin, n) if kin else np.empty(0, dtype=np.uint32)
+        mo = oracle_mod.random_mask(d_out, kout, n + 50) if kout else np.empty(0, dtype=np.uint32)
+        layers.append(dict(A=A, G=Gt, mask_in=_dev_mask(G, mi), mask_out=_dev_mask(G, mo), k=k, s=1, seed=n,
+                           out_offset=off))
+        refs.append((off, k, n, mi, mo, A, Gt))
+        off += k
+    out = torch.full((B, off), 7.0, device="cuda")
+    ws = torch.empty(G.factgrass_grouped_workspace_bytes(len(specs)), dtype=torch.uint8, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    G.factgrass_compress_grouped(G.GroupedLayers(layers), out, ws, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    host = out.cpu().numpy()
+    for (o, k, seed, mi, mo, A, Gt) in refs:
+        if mi.size == 0 or mo.size == 0:
+            assert np.all(host[:, o:o + k] == 0.0)
+            continue
+        ref, absum = oracle_mod.factgrass(W.bits_of(A), W.bits_of(Gt), mi, mo, k, 1, seed)
+        check_close(host[:, o:o + k], ref, absum, TOL_BF16, T + 64, eps=EPS_TC, what=f"empty-mask group off={o}")
+
+
 # ------------------------------------------------------------------ grass_score
 
 @pytest.mark.parametrize("N,M,D", [(300, 70, 257), (128, 128, 64), (1, 1, 1), (513, 256, 4096), (5, 3, 10),
@@ -470,14 +499,14 @@ def test_grass_score_strided_and_compressed_inputs(G, W, oracle_mod):
     check_close(sc, ref, absum, TOL_F32, 520, what="score of compressed")
 
 
-def test_grass_score_split_contraction(G, W, oracle_mod, monkeypatch):
+def test_grass_score_split_contraction(G, W, oracle_mod, tune):
     """The contraction split over several CTAs per output tile (partial products added into the zeroed output):
-    forced through the environment switch, with a ragged last split, vector and scalar reductions (output row
+    forced through the tuning hook, with a ragged last split, vector and scalar reductions (output row
     stride a multiple of four floats or not), stale data in the output buffer; then the two automatic cases,
     a long contraction (D > 16,384) and a small output that would leave most SMs idle."""
     for splits, (N, M, D), ld_s in [(3, (300, 70, 260), 70), (5, (129, 257, 1000), 260), (2, (256, 256, 64), 256),
                                     (64, (40, 300, 128), 301), (7, (513, 24, 4096), 24)]:
-        monkeypatch.setenv("GRASS_SCORE_SPLITS", str(splits))
+        tune(score_splits=splits)
         tr, te = W.score_vectors(N, M, D, 55 + splits, device="cuda")
         buf = torch.full((N, ld_s), 123.0, device="cuda")
         sc = G.grass_score(tr, te, out=buf[:, :M])
@@ -485,7 +514,7 @@ def test_grass_score_split_contraction(G, W, oracle_mod, monkeypatch):
         check_close(sc.cpu().numpy(), ref, absum, TOL_F32, D + 8 + splits, what=f"score {N}x{M}x{D}, {splits} splits")
         if ld_s > M:
             assert torch.all(buf[:, M:] == 123.0), "columns beyond M must not be touched"
-    monkeypatch.delenv("GRASS_SCORE_SPLITS")
+    tune(score_splits=None)
     for (N, M, D) in [(200, 100, 20_000), (64, 32, 8_192), (300, 520, 3_000)]:
         tr, te = W.score_vectors(N, M, D, 77, device="cuda")
         sc = G.grass_score(tr, te, out=torch.full((N, M), -5.0, device="cuda"))

@@ -55,17 +55,17 @@ def test_score_bf16_parity(G, oracle_mod, N, M, D):
     assert torch.all(buf[:, M:] == 9.0)
 
 
-def test_score_bf16_forced_splits_and_unsupported_strides(G, oracle_mod, monkeypatch):
+def test_score_bf16_forced_splits_and_unsupported_strides(G, oracle_mod, tune):
     g = torch.Generator(device="cuda")
     g.manual_seed(3)
     tr = torch.randn((260, 1_000), generator=g, device="cuda").to(torch.bfloat16)
     te = torch.randn((90, 1_000), generator=g, device="cuda").to(torch.bfloat16)
     ref, absum = oracle_mod.score(tr.float().cpu().numpy(), te.float().cpu().numpy())
     for splits in (1, 3, 32):
-        monkeypatch.setenv("GRASS_SCORE_SPLITS", str(splits))
+        tune(score_splits=splits)
         sc = G.grass_score_bf16(tr, te, out=torch.full((260, 90), -1.0, device="cuda"))
         check_close(sc.cpu().numpy(), ref, absum, 1e-4, 1_000 + 72, eps=EPS_TC, what=f"bf16 score, {splits} splits")
-    monkeypatch.delenv("GRASS_SCORE_SPLITS")
+    tune(score_splits=None)
     with pytest.raises(G.GrassError) as e:
         G.grass_score_bf16(tr[:, :996][:, 1:], te[:, :996][:, 1:])          # base not 16-byte aligned
     assert e.value.code == 3
