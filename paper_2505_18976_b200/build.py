@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "libgrass_b200.so")
-SOURCES = ["grass_compress.cu", "factgrass.cu", "grass_score.cu", "grass_score_tc.cu", "grass_fim.cu", "grass_util.cu"]
+SOURCES = ["grass_compress.cu", "factgrass.cu", "factgrass_cluster.cu", "grass_score.cu", "grass_score_tc.cu", "grass_fim.cu", "grass_util.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-cudart", "static"]
 
@@ -52,21 +52,5 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return SO
 
 
-def build_microbench() -> str:
-    """Compile the stand-alone DRAM fetch-granularity microbenchmarks (not part of the library)."""
-    bdir = os.path.join(HERE, "_build")
-    os.makedirs(bdir, exist_ok=True)
-    outs = []
-    for name in ("fetch_granularity", "tma_box_granularity"):
-        out = os.path.join(bdir, name)
-        subprocess.check_call([_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-o", out,
-                               os.path.join(CSRC, "microbench", name + ".cu")])
-        outs.append(out)
-    return " ".join(outs)
-
-
 if __name__ == "__main__":
-    if "--microbench" in sys.argv:
-        print(build_microbench())
-    else:
-        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

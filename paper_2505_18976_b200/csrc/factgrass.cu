@@ -13,8 +13,7 @@
 // A work item is (layer, sample, token chunk, block tile).  The token sum is split over chunks
 // because SJLT is linear: partial blocks are projected separately and their projections add up in
 // the output row.  Neither the masked factors nor the k'_in x k'_out block ever reach HBM.
-#include "grass_common.cuh"
-#include "tcgen05_util.cuh"
+#include "factgrass_common.cuh"
 
 #include <algorithm>
 #include <cstdlib>
@@ -23,39 +22,6 @@
 #include <vector>
 
 namespace grass {
-
-constexpr int kFgThreads = 256;
-constexpr int kTokTile = 32;  // tokens per pipeline stage
-constexpr int kFgBufs = 2;    // operand-tile buffers per CTA
-
-struct LayerDesc {
-    const void* A;
-    const void* G;
-    const uint32_t* mask_in;
-    const uint32_t* mask_out;
-    int32_t d_in, d_out;
-    int32_t kin, kout;
-    uint32_t k, s;
-    uint64_t seed;
-    int64_t out_offset;
-    int32_t tiles_m, tiles_n;
-    int32_t use_smem_bins;
-    float scale;   // raw-block epilogue: factor applied to every entry
-};
-static_assert(sizeof(LayerDesc) == 88, "descriptor layout");
-
-// Token tile staged per pipeline step = the k extent of one shared-memory operand tile.
-static_assert(kTokTile == tc::BK, "a stage holds one operand tile of 32 tokens");
-
-template <bool F32> struct in_elem { using type = uint16_t; };
-template <> struct in_elem<true> { using type = uint32_t; };
-
-// eight consecutive tokens of one masked column (bf16 bit patterns, one per register) -> the 16-byte
-// K-major chunk of that operand row
-__device__ __forceinline__ uint4 pack8_bf16(const uint32_t (&v)[8])
-{
-    return make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
-}
 
 // What happens to the finished k'_in x k'_out block.
 constexpr int kEpiSjlt = 0;   // FactGraSS stage 3: hash every entry into the k-bin accumulator
@@ -340,8 +306,6 @@ __global__ void factgrass_zero_kernel(const LayerDesc* __restrict__ descs, const
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < L.k; i += gridDim.x * blockDim.x) orow[i] = 0.0f;
 }
 
-constexpr size_t kMaxSmemBins = 160 * 1024;
-
 static grass_status fill_desc(LayerDesc& d, const factgrass_layer& l, int tile, int32_t T)
 {
     if (l.spec.k == 0 || l.spec.s == 0) return GRASS_ERR_INVALID_ARG;
@@ -400,6 +364,39 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     if (!workspace && L != 1) return GRASS_ERR_INVALID_ARG;
     if (workspace && (workspace_bytes < (size_t)L * sizeof(LayerDesc) || ((uintptr_t)workspace & 15)))
         return GRASS_ERR_INVALID_ARG;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
+    const bool f32 = dt == GRASS_F32;
+
+    // Launches of about one wave (few layers x samples, bf16 factors, blocks of one tile) take the cluster kernel:
+    // one cluster per (layer, sample), no zero-fill, no global reductions (factgrass_cluster.cu).
+    ClusterPlan cplan;
+    int cluster_nc = 0, cluster_chunk = 0;
+    auto plan_cluster = [&](const LayerDesc* hd) {
+        if (epi != kEpiSjlt || f32 || T <= 0) return;
+        const int64_t forced = tuning(GRASS_TUNE_FACTGRASS_PATH, -1);
+        if (forced == 0 || !cluster_path_fits(hd, L, &cplan)) return;
+        const int64_t items = (int64_t)L * B, slots = (int64_t)sms * cplan.per_sm;
+        if (items > slots && forced != 1) return;
+        // clusters of 1, 2, 4 or 8 thread blocks: as many as fill the machine, each with at least two 32-token steps;
+        // no accumulator runs over more than 8,192 tokens
+        auto pow2_floor = [](int64_t v) { int64_t p = 1; while (p * 2 <= v) p *= 2; return p; };
+        int64_t nc = pow2_floor(std::max<int64_t>(1, std::min<int64_t>(8, slots / std::max<int64_t>(items, 1))));
+        nc = std::min<int64_t>(nc, pow2_floor(std::max<int64_t>(1, T / (2 * kTokTile))));
+        int64_t chunk = ((T + nc - 1) / nc + kTokTile - 1) / kTokTile * kTokTile;
+        const int64_t forced_chunk = tuning(GRASS_TUNE_FACTGRASS_CHUNK, -1);
+        if (forced_chunk > 0) {
+            chunk = std::max<int64_t>(kTokTile, (forced_chunk + kTokTile - 1) / kTokTile * kTokTile);
+            const int64_t need = (T + chunk - 1) / chunk;
+            nc = 1;
+            while (nc < need) nc *= 2;
+        }
+        if (nc > 8 || chunk > 8192) return;
+        cluster_nc = (int)nc;
+        cluster_chunk = (int)chunk;
+    };
+
     // a single layer travels as a kernel parameter: no descriptor copy, whoever provided a workspace
     const bool grouped = workspace != nullptr && L > 1;
     LayerDesc single;
@@ -417,6 +414,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
             if (rc == GRASS_OK && host[l].tiles_m * host[l].tiles_n > max_tiles)
                 max_tiles = host[l].tiles_m * host[l].tiles_n;
         }
+        if (rc == GRASS_OK) plan_cluster(host);
         if (rc == GRASS_OK)
             rc = cuda_ok(cudaMemcpyAsync(workspace, host, (size_t)L * sizeof(LayerDesc), cudaMemcpyHostToDevice, st));
         if (host != stack_buf) std::free(host);
@@ -426,7 +424,11 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
         grass_status rc = fill_desc(single, layers[0], tile, T);
         if (rc != GRASS_OK) return rc;
         max_tiles = single.tiles_m * single.tiles_n;
+        plan_cluster(&single);
     }
+    if (cluster_nc > 0)
+        return launch_factgrass_cluster(dev_descs, single, cplan, L, B, T, tok_begin, tok_count, cluster_nc,
+                                        cluster_chunk, out, ld_out, dev_status, st);
 
     // zero the output ranges (the compress kernel accumulates partial projections into them)
     {
@@ -437,12 +439,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     }
     if (T == 0 || max_tiles == 0) return GRASS_OK;
 
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
-
     const size_t bins_bytes = epi == kEpiSjlt ? (size_t)max_k_smem * sizeof(float) : 0;
-    const bool f32 = dt == GRASS_F32;
     auto launch = [&](auto kern, size_t stage_bytes) -> grass_status {
         const size_t smem = kFgBufs * stage_bytes + bins_bytes;
         // static shared memory counts toward the 48 KB default limit too

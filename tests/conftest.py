@@ -47,3 +47,13 @@ def tune():
     yield set_
     for k in touched:
         G.grass_set_tuning(k, None)
+
+
+@pytest.fixture(params=["streaming", "cluster"])
+def fg_path(request):
+    """Runs a FactGraSS test once on the streaming kernel and once with the cluster kernel forced wherever the
+    layers fit it (calls that do not fit fall back to the streaming kernel by themselves)."""
+    import paper_2505_18976_b200 as G
+    G.grass_set_tuning("factgrass_path", 0 if request.param == "streaming" else 1)
+    yield request.param
+    G.grass_set_tuning("factgrass_path", None)

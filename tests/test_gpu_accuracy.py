@@ -59,8 +59,10 @@ def test_score_single_accumulator_accuracy(G, W, oracle_mod, tune, D):
     tr, te = W.score_vectors(384, 256, D, 5, device="cuda")
     sc = G.grass_score(tr, te).cpu().numpy()
     ref, absum = oracle_mod.score(tr.cpu().numpy(), te.cpu().numpy())
+    # `rel` covers outputs down to |ref| = 2^-10 absum, where a sum of D signed terms has lost two to three
+    # digits to cancellation: it is bounded loosely here, the arithmetic itself by assert_accurate
     rel = check_close(sc, ref, absum, 1e-4, D + 8, what=f"score D={D}, one accumulator")
-    assert rel <= 1e-4
+    assert rel <= 1e-3
     assert_accurate(sc, ref, 2e-5, what=f"score D={D}, one accumulator")
 
 
@@ -90,18 +92,37 @@ def test_fim_accuracy_at_n_4096(G, oracle_mod):
     F = G.grass_fim(X).cpu().numpy()
     ref, absum = oracle_mod.fim(X.cpu().numpy())
     rel = check_close(F, ref, absum, 1e-4, 4096 + 64, eps=2.0 ** -23, what="fim n=4096")
-    assert rel <= 1e-4
+    assert rel <= 1e-3
     assert_accurate(F, ref, 2e-5, what="fim n=4096")
 
 
-@pytest.mark.parametrize("nprod,limit", [(4, 4e-6), (3, 2e-5)])
+@pytest.mark.parametrize("nprod,limit", [(4, 4e-6), (3, 4e-6)])
 def test_fewer_partial_products_stay_unbiased(G, oracle_mod, tune, nprod, limit):
-    """The pieces are rounded to nearest, so what two pieces leave out has either sign: with four products
-    (no lo piece at all) sums over operands of one sign are still right to a few 1e-6, and with three (mid*mid
-    dropped as well, a term of one sign at 2^-18 .. 2^-16) to about 1e-5.  Six stay the default: they make every
-    single product fp32-accurate, these only the sums."""
+    """The pieces are rounded to nearest, so what two pieces leave out has either sign (at most 2^-17 of a
+    product): with four products (no lo piece at all), and with three (mid*mid dropped as well), sums over
+    operands of one sign are still right to about 1e-6.  Six stay the default: they make every single product
+    fp32-accurate, these only the sums, and the kernels' time does not depend on the count (the split of the
+    operands sets the pace, not the tensor pipe)."""
     tr, te = _positive((300, 512), 1), _positive((70, 512), 2)
     ref, _ = oracle_mod.score(tr.cpu().numpy(), te.cpu().numpy())
     tune(score_splits=1, split_products=nprod)
     rel = _max_rel(G.grass_score(tr, te).cpu().numpy(), ref)
     assert rel <= limit, (nprod, rel)
+
+
+def test_worst_case_operands_show_what_the_last_two_products_buy(G, tune):
+    """x = 1 + 2^-9 + 2^-18 in every entry: the third bf16 piece of each operand is 2^-18 with the same sign
+    everywhere, so dropping it (four products) errs by 2 * 2^-18 = 7.6e-6 of every product and of their sum
+    (closed form D x^2); all six products leave only the accumulator's truncation."""
+    x = 1.0 + 2.0 ** -9 + 2.0 ** -18
+    D = 512
+    tr = torch.full((256, D), x, device="cuda")
+    te = torch.full((64, D), x, device="cuda")
+    assert float(tr[0, 0].double().item()) == x                      # exact in fp32
+    exact = D * x * x
+    tune(score_splits=1)
+    rel6 = float((G.grass_score(tr, te).double() - exact).abs().max().item() / exact)
+    assert rel6 <= 4e-6, rel6
+    tune(split_products=4)
+    rel4 = float((G.grass_score(tr, te).double() - exact).abs().max().item() / exact)
+    assert 5e-6 <= rel4 <= 2e-5, rel4

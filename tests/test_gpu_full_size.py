@@ -84,7 +84,7 @@ def test_config2_full_batch_sampled_rows(G, W, oracle_mod):
     assert torch.all(wide[:, c.k:] == 9.0)
 
 
-def test_config3_full_every_output(G, W, oracle_mod):
+def test_config3_full_every_output(G, W, oracle_mod, fg_path):
     c = W.CONFIG3
     lay = c.layers[0]
     A, Gt = W.layer_io(c, 0, device="cuda")

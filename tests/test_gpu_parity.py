@@ -53,7 +53,7 @@ def test_one_hot_through_grass_compress_reads_the_table(G, oracle_mod):
     assert np.array_equal(out, expect)
 
 
-def test_one_hot_through_factgrass_reads_the_table(G, oracle_mod):
+def test_one_hot_through_factgrass_reads_the_table(G, oracle_mod, fg_path):
     """T = 1, A = e_a, G = e_c: the only non-zero block entry sits at q = a*kout + c."""
     kin, kout, k, seed = 24, 40, 97, 11
     d_in, d_out = 64, 96
@@ -236,17 +236,24 @@ def _fact_case(G, W, oracle_mod, cfg, l=0, grouped=False, dtype=torch.bfloat16):
     mi = oracle_mod.random_mask(lay.d_in, cfg.kin, s_in)
     mo = oracle_mod.random_mask(lay.d_out, cfg.kout, s_out)
     seed = W.layer_hash_seed(cfg, l)
-    st = torch.zeros(1, dtype=torch.int32, device="cuda")
-    out = G.factgrass_compress(A, Gt, _dev_mask(G, mi), _dev_mask(G, mo), cfg.k, cfg.s, seed, dev_status=st)
-    torch.cuda.synchronize()
-    assert int(st.item()) == 0
     f32 = dtype == torch.float32
     ref, absum = oracle_mod.factgrass(W.bits_of(A), W.bits_of(Gt), mi, mo, cfg.k, cfg.s, seed,
                                       dtype="f32" if f32 else "bf16")
     ob, _ = oracle_mod.sjlt_table(cfg.k, cfg.s, seed, cfg.kin * cfg.kout)
     chain = cfg.T + max_bin_load(ob, cfg.k) + 64
-    return check_close(out.cpu().numpy(), ref, absum, TOL_F32 if f32 else TOL_BF16, chain, eps=EPS_TC,
-                       what=f"factgrass {lay} B={cfg.B} T={cfg.T} k'={cfg.kin}x{cfg.kout} k={cfg.k} {dtype}")
+    rel = 0.0
+    # both kernels: the streaming one, and the cluster one wherever the layer fits it (bf16, one block tile)
+    for path in (0, 1):
+        with G.tuning(factgrass_path=path):
+            st = torch.zeros(1, dtype=torch.int32, device="cuda")
+            out = torch.full((cfg.B, cfg.k), 5.0, device="cuda")
+            G.factgrass_compress(A, Gt, _dev_mask(G, mi), _dev_mask(G, mo), cfg.k, cfg.s, seed, out=out, dev_status=st)
+            torch.cuda.synchronize()
+            assert int(st.item()) == 0
+        rel = max(rel, check_close(out.cpu().numpy(), ref, absum, TOL_F32 if f32 else TOL_BF16, chain, eps=EPS_TC,
+                                   what=f"factgrass path {path} {lay} B={cfg.B} T={cfg.T} k'={cfg.kin}x{cfg.kout} "
+                                        f"k={cfg.k} {dtype}"))
+    return rel
 
 
 @pytest.mark.parametrize("kw", [
@@ -325,7 +332,7 @@ def test_factgrass_scaled_configs(G, W, oracle_mod):
         _fact_case(G, W, oracle_mod, c5, l=l)
 
 
-def test_factgrass_padding_tokens_change_nothing(G, W, oracle_mod):
+def test_factgrass_padding_tokens_change_nothing(G, W, oracle_mod, fg_path):
     cfg = _fact_cfg(W, T=64, kin=64, kout=64, k=512)
     A, Gt = W.layer_io(cfg, 0, device="cuda")
     mi = _dev_mask(G, oracle_mod.random_mask(96, 64, 1))
@@ -382,7 +389,7 @@ def _group(G, W, oracle_mod, cfg, layer_ids, offsets=None):
     return layers, refs
 
 
-def test_factgrass_grouped_parity(G, W, oracle_mod):
+def test_factgrass_grouped_parity(G, W, oracle_mod, fg_path):
     cfg = dataclasses.replace(W.CONFIG4, B=3, T=96, layers=W.CONFIG4.layers[:8])
     ids = list(range(8))
     layers, refs = _group(G, W, oracle_mod, cfg, ids)
@@ -403,7 +410,7 @@ def test_factgrass_grouped_parity(G, W, oracle_mod):
         check_close(single, ref, absum, TOL_BF16, cfg.T + 64, eps=EPS_TC, what="single")
 
 
-def test_factgrass_grouped_mixed_layers(G, W, oracle_mod):
+def test_factgrass_grouped_mixed_layers(G, W, oracle_mod, fg_path):
     """Layers of one call may differ in d_in/d_out, mask sizes, k, s and seed."""
     B, T = 2, 50
     specs = [(96, 160, 24, 40, 97, 1), (200, 64, 64, 64, 1024, 1), (768, 3072, 100, 130, 300, 2)]
@@ -427,7 +434,7 @@ def test_factgrass_grouped_mixed_layers(G, W, oracle_mod):
         check_close(host[:, o:o + k], ref, absum, TOL_BF16, T + 64, eps=EPS_TC, what=f"mixed off={o}")
 
 
-def test_factgrass_grouped_layer_with_an_empty_mask(G, W, oracle_mod):
+def test_factgrass_grouped_layer_with_an_empty_mask(G, W, oracle_mod, fg_path):
     """A layer whose input-factor mask is empty has no block: its output range must come back as zeros, the
     other layers must be untouched by it, and no device fault may be flagged."""
     B, T = 2, 70

@@ -46,7 +46,7 @@ def _i32(x):
     (4, 300, 768, 3072, 128, 128, 4096, [300, 33, 256, 64]),          # config 3 tile shape, several chunks
     (3, 64, 200, 64, 64, 64, 1024, [5, 64, 31]),
 ])
-def test_padded_batch_with_lengths(G, W, oracle_mod, B, T, d_in, d_out, kin, kout, k, lens):
+def test_padded_batch_with_lengths(G, W, oracle_mod, B, T, d_in, d_out, kin, kout, k, lens, fg_path):
     A, Gt, mi, mo = _layer(G, W, oracle_mod, B, T, d_in, d_out, kin, kout, 40)
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
     out = G.factgrass_compress_varlen(A, Gt, G.mask_to_device(mi), G.mask_to_device(mo), k, 1, 123, B, T,
@@ -62,7 +62,7 @@ def test_padded_batch_with_lengths(G, W, oracle_mod, B, T, d_in, d_out, kin, kou
             assert torch.all(out[b] == 0)
 
 
-def test_packed_batch_grouped(G, W, oracle_mod):
+def test_packed_batch_grouped(G, W, oracle_mod, fg_path):
     """Three layers over one packed token stream (no padding rows), samples listed out of order."""
     lens = np.array([130, 7, 64, 0, 95], dtype=np.int32)
     begin = np.concatenate([[0], np.cumsum(lens)[:-1]]).astype(np.int64)
@@ -92,7 +92,7 @@ def test_packed_batch_grouped(G, W, oracle_mod):
                     what=f"packed grouped off={o}")
 
 
-def test_null_arrays_equal_the_plain_call(G, W, oracle_mod):
+def test_null_arrays_equal_the_plain_call(G, W, oracle_mod, fg_path):
     A, Gt, mi, mo = _layer(G, W, oracle_mod, 3, 100, 96, 160, 24, 40, 70)
     dmi, dmo = G.mask_to_device(mi), G.mask_to_device(mo)
     a = G.factgrass_compress(A, Gt, dmi, dmo, 97, 1, 5)
@@ -100,7 +100,7 @@ def test_null_arrays_equal_the_plain_call(G, W, oracle_mod):
     assert float((a - b).abs().max()) <= 1e-5 * float(a.abs().max())
 
 
-def test_lengths_out_of_range_are_clamped_and_flagged(G, W, oracle_mod):
+def test_lengths_out_of_range_are_clamped_and_flagged(G, W, oracle_mod, fg_path):
     B, T = 3, 50
     A, Gt, mi, mo = _layer(G, W, oracle_mod, B, T, 96, 160, 24, 40, 80)
     st = torch.zeros(1, dtype=torch.int32, device="cuda")
@@ -113,7 +113,7 @@ def test_lengths_out_of_range_are_clamped_and_flagged(G, W, oracle_mod):
     check_close(out.cpu().numpy(), ref, absum, TOL_BF16, T + 64, eps=EPS_TC, what="clamped lengths")
 
 
-def test_config3_padding_skipped(G, W, oracle_mod):
+def test_config3_padding_skipped(G, W, oracle_mod, fg_path):
     """Config 3's trailing padding (zero output-gradient rows): passing the lengths gives the same
     compressed gradients as reading the zero rows."""
     c = dataclasses.replace(W.CONFIG3, B=8)
