@@ -305,7 +305,7 @@ typedef enum {
     GRASS_TUNE_SCORE_SPLITS = 8,       /* grass_score, grass_score_bf16: splits of the contraction */
     GRASS_TUNE_SPLIT_PRODUCTS = 9,     /* fp32 contractions: partial products per fp32 product (3, 4 or 6) */
     GRASS_TUNE_FACTGRASS_PATH = 10,    /* factgrass: 0 = streaming kernel, 1 = cluster kernel (see factgrass.cu) */
-    GRASS_TUNE_FACTGRASS_STAGING = 11, /* factgrass cluster kernel: 0 = element gathers, 1 = whole token rows staged by TMA */
+    GRASS_TUNE_COMPRESS_ROWS = 11,     /* grass_compress: 0 = never stage row segments in shared memory, 1 = wherever the operands allow */
     GRASS_TUNE_COMPRESS_LOADS = 12,    /* grass_compress gather path: loads in flight per thread (4, 8, 16) */
     GRASS_TUNE_COMPRESS_THREADS = 13,  /* grass_compress gather path: threads per block (256, 512) */
     GRASS_TUNE_COUNT = 14

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "libgrass_b200.so")
-SOURCES = ["grass_compress.cu", "factgrass.cu", "factgrass_cluster.cu", "grass_score.cu", "grass_score_tc.cu", "grass_fim.cu", "grass_util.cu"]
+SOURCES = ["grass_compress.cu", "grass_compress_rows.cu", "factgrass.cu", "factgrass_cluster.cu", "grass_score.cu", "grass_score_tc.cu", "grass_fim.cu", "grass_util.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-cudart", "static"]
 

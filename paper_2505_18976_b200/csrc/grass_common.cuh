@@ -65,6 +65,9 @@ __device__ __forceinline__ uint16_t gather_u16(const uint16_t* p)
     return v;
 }
 
+__device__ __forceinline__ float elem_value(float x) { return x; }
+__device__ __forceinline__ float elem_value(__nv_bfloat16 x) { return __bfloat162float(x); }
+
 template <typename T> struct elem;
 template <> struct elem<float> {
     static __device__ __forceinline__ float load(const float* p)
@@ -78,6 +81,14 @@ template <> struct elem<__nv_bfloat16> {
         return bf16_bits_to_float(gather_u16(reinterpret_cast<const uint16_t*>(p)));
     }
 };
+
+// grass_compress with row staging for dense masks (grass_compress_rows.cu): whether the operands allow it, and
+// the launch
+bool compress_rows_fits(const void* g, size_t elem_bytes, int64_t p, int64_t ld, const uint32_t* idx, int64_t kprime,
+                        uint32_t k, int64_t n);
+grass_status launch_compress_rows(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld, const uint32_t* idx,
+                                  int64_t kprime, const grass_sjlt_spec& sp, float* out, int64_t ld_out,
+                                  uint32_t* dev_status, cudaStream_t st);
 
 // launch-shape override set through grass_set_tuning, or `dflt` while the key is on automatic
 int64_t tuning(grass_tuning_key key, int64_t dflt);

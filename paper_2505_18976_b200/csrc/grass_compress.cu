@@ -42,8 +42,9 @@ __device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&v)[4])
 
 // DENSE: identity mask on vector-aligned rows (plain SJLT, the k' = p case of Section 3.3.1).  Rows are then
 // streamed with vector loads, four consecutive positions per thread, and S > 1 samples share each hash.
-template <typename T, int S, int U, bool S1, bool DENSE>
-__global__ void __launch_bounds__(kThreads, DENSE ? 4 : 0)
+// NT: threads per CTA (the gather path runs with 256 or 512; the streamed path always with kThreads).
+template <typename T, int S, int U, bool S1, bool DENSE, int NT>
+__global__ void __launch_bounds__(NT, DENSE ? 4 : 0)
 grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
                       const uint32_t* __restrict__ idx, int64_t kprime, uint32_t k, uint32_t s,
                       uint64_t seed, float scale, float* __restrict__ out, int64_t ld_out,
@@ -51,13 +52,15 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
 {
     extern __shared__ float bins[];  // S * k when use_smem
     const int tid = threadIdx.x;
+    constexpr int nthr = NT;
+    static_assert(!DENSE || NT == kThreads, "the streamed path is written for kThreads threads");
     const int64_t i0 = (int64_t)blockIdx.x * S;
     const int ns = (int)((n - i0) < (int64_t)S ? (n - i0) : (int64_t)S);
     const int64_t j0 = (int64_t)blockIdx.y * j_per_cta;
     const int64_t j1 = (j0 + j_per_cta) < kprime ? (j0 + j_per_cta) : kprime;
 
     if (use_smem) {
-        for (uint32_t i = tid; i < (uint32_t)S * k; i += kThreads) bins[i] = 0.0f;
+        for (uint32_t i = tid; i < (uint32_t)S * k; i += nthr) bins[i] = 0.0f;
         __syncthreads();
     }
 
@@ -179,12 +182,12 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
             }
         }
     } else
-    for (int64_t jb = j0 + tid; jb < j1; jb += (int64_t)kThreads * U) {
+    for (int64_t jb = j0 + tid; jb < j1; jb += (int64_t)nthr * U) {
         uint32_t col[U];
         bool ok[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int64_t j = jb + (int64_t)u * kThreads;
+            const int64_t j = jb + (int64_t)u * nthr;
             ok[u] = j < j1;
             uint32_t c = 0;
             if (ok[u]) c = idx ? __ldg(idx + j) : (uint32_t)j;
@@ -207,7 +210,7 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
 #pragma unroll
             for (int si = 0; si < S; ++si) any = any || (v[u][si] != 0.0f);
             if (!any) continue;
-            const uint64_t j = (uint64_t)(jb + (int64_t)u * kThreads);
+            const uint64_t j = (uint64_t)(jb + (int64_t)u * nthr);
             const uint32_t draws = S1 ? 1u : s;
             for (uint32_t r = 0; r < draws; ++r) {
                 const uint64_t h = sjlt_hash_counter(seed, S1 ? (j + 1) : (j * s + r + 1));
@@ -236,7 +239,7 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
         const uint32_t lo = r * per, hi = (lo + per) < k ? (lo + per) : k;
         for (int si = 0; si < ns; ++si) {
             float* dst = out + (i0 + si) * ld_out;
-            for (uint32_t i = lo + tid; i < hi; i += kThreads) {
+            for (uint32_t i = lo + tid; i < hi; i += nthr) {
                 float acc = 0.0f;
                 for (uint32_t q = 0; q < nr; ++q) acc += cluster.map_shared_rank(bins, q)[(uint32_t)si * k + i];
                 dst[i] = acc;
@@ -249,12 +252,12 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
             float* dst = out + (i0 + si) * ld_out;
             const float* src = bins + (uint32_t)si * k;
             if (accumulate) {
-                for (uint32_t i = tid; i < k; i += kThreads) {
+                for (uint32_t i = tid; i < k; i += nthr) {
                     const float x = src[i];
                     if (x != 0.0f) atomicAdd(dst + i, x);
                 }
             } else {
-                for (uint32_t i = tid; i < k; i += kThreads) dst[i] = src[i];
+                for (uint32_t i = tid; i < k; i += nthr) dst[i] = src[i];
             }
         }
     }
@@ -285,6 +288,8 @@ struct CompressPlan {
     int jsplit;     // CTAs that share one sample group (split of the masked positions)
     int use_smem;   // k-bin accumulators fit in shared memory
     int cluster;    // the jsplit CTAs are one thread-block cluster (DSMEM reduction)
+    int threads;    // threads per CTA of the gather path (256 or 512)
+    int U;          // gathered loads in flight per thread and sample
 };
 
 static CompressPlan plan_compress(int64_t n, int64_t kprime, uint32_t k, int sm_count, bool dense)
@@ -303,10 +308,14 @@ static CompressPlan plan_compress(int64_t n, int64_t kprime, uint32_t k, int sm_
     while (S > 1 && pl.use_smem && bin_bytes * S > smem_cap) S >>= 1;
     if (!pl.use_smem) S = 1;
     pl.S = S;
-    const int U = S == 1 ? 8 : (S == 8 ? 2 : 4);
+    int U = S == 1 ? 8 : (S == 8 ? 2 : 4);
+    if (S == 1 && !dense && tuning(GRASS_TUNE_COMPRESS_LOADS, 8) == 16) U = 16;
+    pl.U = U;
+    pl.threads = (!dense && tuning(GRASS_TUNE_COMPRESS_THREADS, kThreads) == 2 * kThreads) ? 2 * kThreads : kThreads;
     const int64_t groups = (n + S - 1) / S;
     // split positions until there are ~4 CTAs per SM, but keep one full round of loads per CTA
-    const int64_t max_js = kprime / ((int64_t)kThreads * U) > 0 ? kprime / ((int64_t)kThreads * U) : 1;
+    const int64_t round = (int64_t)pl.threads * U;
+    const int64_t max_js = kprime / round > 0 ? kprime / round : 1;
     int64_t js = 1;
     while (js < 8 && groups * js < (int64_t)sm_count * 4 && js * 2 <= max_js) js *= 2;
     pl.cluster = 1;
@@ -348,7 +357,7 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
         }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)groups, (unsigned)pl.jsplit, 1);
-        cfg.blockDim = dim3(kThreads, 1, 1);
+        cfg.blockDim = dim3((unsigned)(pl.dense ? kThreads : pl.threads), 1, 1);
         cfg.dynamicSmemBytes = smem;
         cfg.stream = st;
         cudaLaunchAttribute attr[1];
@@ -366,11 +375,15 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
         return e == cudaSuccess ? launch_status() : GRASS_ERR_CUDA;
     };
     if (pl.dense) {
-        if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true, true>);
-        return launch(grass_compress_kernel<T, S, U, false, true>);
+        if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true, true, kThreads>);
+        return launch(grass_compress_kernel<T, S, U, false, true, kThreads>);
     }
-    if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true, false>);
-    return launch(grass_compress_kernel<T, S, U, false, false>);
+    if (pl.threads == 2 * kThreads) {
+        if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true, false, 2 * kThreads>);
+        return launch(grass_compress_kernel<T, S, U, false, false, 2 * kThreads>);
+    }
+    if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true, false, kThreads>);
+    return launch(grass_compress_kernel<T, S, U, false, false, kThreads>);
 }
 
 template <typename T>
@@ -393,7 +406,10 @@ static grass_status dispatch_compress(const T* g, int64_t n, int64_t p, int64_t 
         case 8: return launch_compress<T, 8, 2>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
         case 4: return launch_compress<T, 4, 4>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
         case 2: return launch_compress<T, 2, 4>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
-        default: return launch_compress<T, 1, 8>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
+        default:
+            if (pl.U == 16)
+                return launch_compress<T, 1, 16>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
+            return launch_compress<T, 1, 8>(g, n, p, ld, idx, kprime, sp, out, ld_out, pl, dev_status, st);
     }
 }
 
@@ -434,6 +450,15 @@ extern "C" grass_status grass_compress(const void* g, grass_dtype dt, int64_t n,
         return grass::cuda_ok(cudaMemset2DAsync(out, (size_t)ld_out * sizeof(float), 0,
                                                 (size_t)spec->k * sizeof(float), (size_t)n, st));
     }
+    // Row staging for dense masks (grass_compress_rows.cu): whole rows through shared memory, window by window,
+    // the masked elements picked from there.  It is built and parity-tested but not chosen automatically: on B200
+    // it is slower than the gathers below even where the mask touches nine pieces in ten (config 1: 28.6 against
+    // 26.5 us), because the bytes a staging kernel keeps in flight are bounded by shared memory (about 19 MB over
+    // the whole GPU) and that is just the latency-bandwidth product of HBM, while the gather kernel has every
+    // load of the launch in flight at once.  GRASS_TUNE_COMPRESS_ROWS = 1 selects it.
+    if (grass::tuning(GRASS_TUNE_COMPRESS_ROWS, 0) == 1 &&
+        grass::compress_rows_fits(g, dt == GRASS_F32 ? 4 : 2, p, ld, idx, kprime, spec->k, n))
+        return grass::launch_compress_rows(g, dt, n, p, ld, idx, kprime, *spec, out, ld_out, dev_status, st);
     if (dt == GRASS_F32)
         return grass::dispatch_compress<float>((const float*)g, n, p, ld, idx, kprime, *spec, out, ld_out,
                                                dev_status, st);

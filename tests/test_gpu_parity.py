@@ -80,17 +80,24 @@ def _grass_case(G, W, oracle_mod, n, p, kprime, k, s=1, dtype=torch.float32, ld=
     g = W.dense_gradients(n, p, zero_prob, dist, scale, data_seed, device="cuda", dtype=dtype, ld=ld)
     idx = None if identity else oracle_mod.random_mask(p, kprime, seed)
     didx = None if identity else _dev_mask(G, idx)
-    status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    out = G.grass_compress(g, didx, k, s, seed + 99, p=p, dev_status=status)
-    torch.cuda.synchronize()
-    assert int(status.item()) == 0
     host = W.bits_of(g)
     ref, absum = oracle_mod.grass(host, idx, k, s, seed + 99, dtype="f32" if dtype == torch.float32 else "bf16", p=p)
     kp = p if identity else kprime
     ob, _ = oracle_mod.sjlt_table(k, s, seed + 99, kp)
     chain = max_bin_load(ob, k) + 16
-    return check_close(out.cpu().numpy(), ref, absum, TOL_F32, chain,
-                       what=f"grass n={n} p={p} k'={kp} k={k} s={s}")
+    rel = 0.0
+    # both kernels: element gathers, and whole row segments staged in shared memory wherever the operands allow
+    # (a mask, 16-byte aligned rows, at most 8 segments per row); the launch-shape overrides of a test stay in force
+    for rows in ((0,) if identity else (0, 1)):
+        with G.tuning(compress_rows=rows):
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            out = torch.full((n, k), 7.0, device="cuda")
+            G.grass_compress(g, didx, k, s, seed + 99, out=out, p=p, dev_status=status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+        rel = max(rel, check_close(out.cpu().numpy(), ref, absum, TOL_F32, chain,
+                                   what=f"grass rows={rows} n={n} p={p} k'={kp} k={k} s={s}"))
+    return rel
 
 
 @pytest.mark.parametrize("n,p,kprime,k", [
@@ -194,13 +201,15 @@ def test_grass_compress_empty_and_errors(G, oracle_mod):
     bad = idxh.copy()
     bad[-1] = 2_000_000_000
     g = torch.randn(2, p, device="cuda")
-    st = torch.zeros(1, dtype=torch.int32, device="cuda")
-    got = G.grass_compress(g, G.mask_to_device(bad), k, 1, 5, dev_status=st).cpu().numpy()
-    assert int(st.item()) & 1
     ref_in = g.cpu().numpy().copy()
     ref_in[:, idxh[-1]] = 0        # same as dropping the last masked position
     ref, absum = oracle_mod.grass(ref_in, idxh, k, 1, 5)
-    check_close(got, ref, absum, TOL_F32, 32, what="bad index skipped")
+    for rows in (0, 1):            # the gather kernel and the row-staging kernel
+        with G.tuning(compress_rows=rows):
+            st = torch.zeros(1, dtype=torch.int32, device="cuda")
+            got = G.grass_compress(g, G.mask_to_device(bad), k, 1, 5, dev_status=st).cpu().numpy()
+            assert int(st.item()) & 1
+            check_close(got, ref, absum, TOL_F32, 32, what=f"bad index skipped, rows={rows}")
     assert not G.grass_validate_mask(G.mask_to_device(bad), p)
     assert G.grass_validate_mask(G.mask_to_device(idxh), p)
     dup = idxh.copy()
