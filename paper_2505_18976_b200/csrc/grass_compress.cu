@@ -44,7 +44,7 @@ __device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&v)[4])
 // streamed with vector loads, four consecutive positions per thread, and S > 1 samples share each hash.
 // NT: threads per CTA (the gather path runs with 256 or 512; the streamed path always with kThreads).
 template <typename T, int S, int U, bool S1, bool DENSE, int NT>
-__global__ void __launch_bounds__(NT, DENSE ? 4 : 0)
+__global__ void __launch_bounds__(NT, DENSE ? 4 : (U >= 16 ? 1024 : 2048) / NT)
 grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
                       const uint32_t* __restrict__ idx, int64_t kprime, uint32_t k, uint32_t s,
                       uint64_t seed, float scale, float* __restrict__ out, int64_t ld_out,
@@ -182,7 +182,9 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
             }
         }
     } else
-    for (int64_t jb = j0 + tid; jb < j1; jb += (int64_t)nthr * U) {
+    // the trip count is the same for every lane of a warp (the warp votes below)
+    for (int64_t jw = j0 + (tid & ~31); jw < j1; jw += (int64_t)nthr * U) {
+        const int64_t jb = jw + (tid & 31);
         uint32_t col[U];
         bool ok[U];
 #pragma unroll
@@ -201,27 +203,54 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
             for (int si = 0; si < S; ++si)
                 v[u][si] = (ok[u] && si < ns) ? elem<T>::load(rows[si] + col[u]) : 0.0f;
 
+        if constexpr (S == 1) {
+            // The cost of the projection follows the non-zeros (Section 3.1).  A lane hashes its own non-zero
+            // entries one after the other, so the warp makes as many passes as its fullest lane has non-zeros
+            // (three or four of eight at 90 % zeros) instead of one per loaded entry.
+            uint32_t pending = 0;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (!ok[u]) continue;
-            // the hash is only worth computing where some sample has a non-zero entry (Section 3.1: the cost of
-            // the projection follows the number of non-zeros)
-            bool any = false;
+            for (int u = 0; u < U; ++u) pending |= (ok[u] && v[u][0] != 0.0f) ? (1u << u) : 0u;
+            while (__any_sync(0xFFFFFFFFu, pending != 0)) {
+                if (pending != 0) {
+                    const int u = __ffs((int)pending) - 1;
+                    pending &= pending - 1;
+                    float x = v[0][0];
 #pragma unroll
-            for (int si = 0; si < S; ++si) any = any || (v[u][si] != 0.0f);
-            if (!any) continue;
-            const uint64_t j = (uint64_t)(jb + (int64_t)u * nthr);
-            const uint32_t draws = S1 ? 1u : s;
-            for (uint32_t r = 0; r < draws; ++r) {
-                const uint64_t h = sjlt_hash_counter(seed, S1 ? (j + 1) : (j * s + r + 1));
-                const uint32_t b = sjlt_bucket(h, k);
-#pragma unroll
-                for (int si = 0; si < S; ++si) {
-                    const float x = v[u][si];
-                    if (x != 0.0f) {
+                    for (int t = 1; t < U; ++t) x = (u == t) ? v[t][0] : x;
+                    const uint64_t j = (uint64_t)(jb + (int64_t)u * nthr);
+                    const uint32_t draws = S1 ? 1u : s;
+                    for (uint32_t r = 0; r < draws; ++r) {
+                        const uint64_t h = sjlt_hash_counter(seed, S1 ? (j + 1) : (j * s + r + 1));
+                        const uint32_t b = sjlt_bucket(h, k);
                         const float sx = S1 ? sjlt_signed(h, x) : sjlt_signed(h, x) * scale;
-                        if (use_smem) atomicAdd(&bins[(uint32_t)si * k + b], sx);
-                        else atomicAdd(out + (i0 + si) * ld_out + b, sx);
+                        if (use_smem) atomicAdd(&bins[b], sx);
+                        else atomicAdd(out + i0 * ld_out + b, sx);
+                    }
+                }
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (!ok[u]) continue;
+                // the hash is shared by the samples of the thread block: it is computed where any of them has a
+                // non-zero entry
+                bool any = false;
+#pragma unroll
+                for (int si = 0; si < S; ++si) any = any || (v[u][si] != 0.0f);
+                if (!any) continue;
+                const uint64_t j = (uint64_t)(jb + (int64_t)u * nthr);
+                const uint32_t draws = S1 ? 1u : s;
+                for (uint32_t r = 0; r < draws; ++r) {
+                    const uint64_t h = sjlt_hash_counter(seed, S1 ? (j + 1) : (j * s + r + 1));
+                    const uint32_t b = sjlt_bucket(h, k);
+#pragma unroll
+                    for (int si = 0; si < S; ++si) {
+                        const float x = v[u][si];
+                        if (x != 0.0f) {
+                            const float sx = S1 ? sjlt_signed(h, x) : sjlt_signed(h, x) * scale;
+                            if (use_smem) atomicAdd(&bins[(uint32_t)si * k + b], sx);
+                            else atomicAdd(out + (i0 + si) * ld_out + b, sx);
+                        }
                     }
                 }
             }
