@@ -2,11 +2,12 @@
 
 Two ways in, both through the C ABI on torch's current stream, both returning the compressed rows in host
 memory.  Staged: the inputs are copied to the device on a copy stream, the copy of the next chunk overlapping
-the kernels of the current one (two device staging slots).  In place (``zero_copy``, the default when every
-input is pinned and the masks are sparse): the kernels gather the masked elements straight from the page-locked host buffers, so only
-the 64-byte pieces the masks touch cross the bus instead of every byte of the inputs (chosen when the masks
-touch less than 70 % of the input bytes).  Only marshalling and
-copies happen here; every step of the compression runs in the kernels.
+the kernels of the current one (two device staging slots).  In place (``zero_copy``): the kernels gather the
+masked elements straight from the page-locked host buffers, so only the 64-byte pieces the masks touch cross the
+bus instead of every byte of the inputs.  Left to choose (``zero_copy=None``), the FactGraSS call decides tensor by
+tensor: a factor whose mask touches less than 70 % of its bytes is read in place, a denser one is copied to the
+device first, and one grouped launch takes both kinds of pointers.  Only marshalling and copies happen here;
+every step of the compression runs in the kernels.
 """
 from __future__ import annotations
 
@@ -40,18 +41,28 @@ def grass_in_place(g_chunks: Sequence[torch.Tensor], idx: Optional[np.ndarray]) 
             touched_fraction(idx, int(g_chunks[0].shape[1]), g_chunks[0].element_size()) <= IN_PLACE_MAX_FRACTION)
 
 
-def factgrass_in_place(groups: Sequence[Sequence[dict]]) -> bool:
-    """Whether factgrass_compress_host, left to choose, gathers from the host buffers in place."""
-    if not all(l["A"].is_pinned() and l["G"].is_pinned() for g in groups for l in g):
-        return False
-    moved = total = 0.0
+def factgrass_host_plan(groups: Sequence[Sequence[dict]]):
+    """What factgrass_compress_host does when left to choose: per layer (A in place?, G in place?), and the bytes
+    that cross the bus (whole tensors that are copied + the 64-byte pieces the masks touch of the others; a host
+    count, not a bus counter)."""
+    plan, moved = [], 0.0
     for g in groups:
         for l in g:
+            dec = []
             for t, m in ((l["A"], l["mask_in"]), (l["G"], l["mask_out"])):
                 nbytes = t.numel() * t.element_size()
-                total += nbytes
-                moved += nbytes * touched_fraction(m, int(t.shape[-1]), t.element_size())
-    return moved <= IN_PLACE_MAX_FRACTION * total
+                frac = touched_fraction(m, int(t.shape[-1]), t.element_size())
+                in_place = bool(t.is_pinned() and frac <= IN_PLACE_MAX_FRACTION)
+                moved += nbytes * (frac if in_place else 1.0)
+                dec.append(in_place)
+            plan.append(tuple(dec))
+    return plan, int(moved)
+
+
+def factgrass_in_place(groups: Sequence[Sequence[dict]]) -> bool:
+    """Whether factgrass_compress_host, left to choose, reads at least one tensor in place."""
+    plan, _ = factgrass_host_plan(groups)
+    return any(a or g for a, g in plan)
 
 
 def grass_compress_host(g_chunks: Sequence[torch.Tensor], idx: np.ndarray, k: int, s: int, seed: int,
@@ -133,10 +144,19 @@ def factgrass_compress_host(groups: Sequence[Sequence[dict]], Bsz: int, T: int, 
         return masks[key]
 
     if zero_copy is None:
-        zero_copy = factgrass_in_place(groups)
+        plan, _ = factgrass_host_plan(groups)
+        zero_copy = any(a or g for a, g in plan)
+    elif zero_copy:
+        plan = [(True, True) for g in groups for l in g]
     if zero_copy:
-        flat = [dict(A=l["A"], G=l["G"], mask_in=dev_mask(l["mask_in"]), mask_out=dev_mask(l["mask_out"]),
-                     k=l["k"], s=l["s"], seed=l["seed"], out_offset=l["out_offset"]) for g in groups for l in g]
+        # tensors that are not read in place are copied to the device first (same stream: the kernels that gather
+        # across the bus would compete with the copies for it anyway)
+        def operand(t, in_place):
+            return t if in_place else t.to(device, non_blocking=True)
+        layers = [l for g in groups for l in g]
+        flat = [dict(A=operand(l["A"], pa), G=operand(l["G"], pg), mask_in=dev_mask(l["mask_in"]),
+                     mask_out=dev_mask(l["mask_out"]), k=l["k"], s=l["s"], seed=l["seed"], out_offset=l["out_offset"])
+                for l, (pa, pg) in zip(layers, plan)]
         per_call = 256
         wsz = torch.empty(B.factgrass_grouped_workspace_bytes(min(per_call, len(flat))), dtype=torch.uint8,
                           device=device)

@@ -113,6 +113,12 @@ def test_config4_block_in_place_matches_device_resident(G, W, oracle_mod):
         dev_layers.append(dict(A=A, G=Gt, mask_in=G.mask_to_device(mi), mask_out=G.mask_to_device(mo), **common))
         host_layers.append(dict(A=_pinned(A.cpu()), G=_pinned(Gt.cpu()), mask_in=mi, mask_out=mo, **common))
     assert host_api.factgrass_in_place([host_layers])
+    # the choice is made tensor by tensor: the 768-wide factors (three in four pieces touched) are copied, the
+    # 2,304- and 3,072-wide ones are gathered in place
+    plan, moved = host_api.factgrass_host_plan([host_layers])
+    flat = [d for pair in plan for d in pair]
+    assert True in flat and False in flat
+    assert moved < sum(l["A"].numel() * 2 + l["G"].numel() * 2 for l in host_layers)
     out_dev = torch.empty((c.B, 4 * c.k), device="cuda")
     ws = torch.empty(G.factgrass_grouped_workspace_bytes(4), dtype=torch.uint8, device="cuda")
     G.factgrass_compress_grouped(G.GroupedLayers(dev_layers), out_dev, ws)
