@@ -133,6 +133,27 @@ grass_status factgrass_compress_grouped(const factgrass_layer* layers /*host*/, 
 size_t factgrass_grouped_workspace_bytes(int32_t L);
 
 /*
+ * The same two compressors writing the compressed rows in a chosen precision (the paper leaves the storage
+ * precision of the cache open; a bf16 cache is half the bytes and feeds grass_score_bf16 directly).
+ *   out_dt   GRASS_F32: identical to grass_compress / factgrass_compress_grouped.
+ *            GRASS_BF16: out is n x k (B x ld_out) bf16, ld_out in elements.  Everything up to the final store is
+ *            the fp32 arithmetic of the fp32 calls; each output is rounded to nearest even exactly once.  That
+ *            needs a launch in which one thread block or one cluster owns a whole row, so there are no partial
+ *            sums in global memory: grass_compress_out then needs k small enough for shared-memory bins (k <=
+ *            51,200); factgrass_compress_grouped_out needs k'_in, k'_out <= 64 (or a launch small enough for the
+ *            cluster kernel: k'_in, k'_out <= 128), T <= 8,192 and k <= 40,960.  Anything else returns
+ *            GRASS_ERR_UNSUPPORTED with nothing enqueued (use the fp32 call and grass_to_bf16).
+ *   factgrass_compress_grouped_out accepts workspace == NULL for a single layer (L == 1).
+ */
+grass_status grass_compress_out(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld,
+                                const uint32_t* idx, int64_t kprime, const grass_sjlt_spec* spec /*host*/,
+                                void* out, grass_dtype out_dt, int64_t ld_out, uint32_t* dev_status, void* stream);
+grass_status factgrass_compress_grouped_out(const factgrass_layer* layers /*host*/, int32_t L, grass_dtype dt,
+                                            int32_t B, int32_t T, void* out, grass_dtype out_dt, int64_t ld_out,
+                                            void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                                            void* stream);
+
+/*
  * Sparsification alone (Section 3.2: Random / Selective Mask used as the whole compressor, which the
  * paper evaluates next to GraSS and FactGraSS).
  *   grass_mask         out[i, j] = g[i, idx[j]],  out n x kprime fp32 (row stride ld_out >= kprime);

@@ -28,7 +28,8 @@ EXPORTS = ("grass_compress", "factgrass_compress", "factgrass_compress_grouped",
            "grass_fim", "grass_fim_factor", "grass_fim_apply", "grass_mask", "factmask_compress",
            "factmask_compress_grouped",
            "factgrass_grouped_workspace_bytes", "factgrass_compress_grouped_static", "grass_score", "grass_sjlt_table", "grass_validate_mask",
-           "grass_random_mask_host", "grass_status_string", "grass_to_bf16", "grass_score_bf16", "grass_set_tuning")
+           "grass_random_mask_host", "grass_status_string", "grass_to_bf16", "grass_score_bf16", "grass_set_tuning",
+           "grass_compress_out", "factgrass_compress_grouped_out")
 
 # grass_tuning_key in include/grass.h
 TUNE = {"compress_samples": 0, "compress_jsplit": 1, "compress_cluster": 2, "compress_dense": 3,
@@ -69,6 +70,11 @@ def lib() -> ctypes.CDLL:
         sp = ctypes.POINTER(SjltSpec)
         L.grass_compress.restype = st
         L.grass_compress.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, i64, sp, vp, i64, vp, vp]
+        L.grass_compress_out.restype = st
+        L.grass_compress_out.argtypes = [vp, ctypes.c_int, i64, i64, i64, vp, i64, sp, vp, ctypes.c_int, i64, vp, vp]
+        L.factgrass_compress_grouped_out.restype = st
+        L.factgrass_compress_grouped_out.argtypes = [ctypes.POINTER(FactgrassLayer), i32, ctypes.c_int, i32, i32, vp,
+                                                     ctypes.c_int, i64, vp, ctypes.c_size_t, vp, vp]
         L.factgrass_compress.restype = st
         L.factgrass_compress.argtypes = [vp, vp, ctypes.c_int, i32, i32, i32, i32, vp, i32, vp, i32, sp, vp, i64, vp, vp]
         L.factgrass_compress_grouped.restype = st
@@ -194,10 +200,11 @@ def _compute_device(t: torch.Tensor) -> torch.device:
 
 def grass_compress(g: torch.Tensor, idx: Optional[torch.Tensor], k: int, s: int, seed: int,
                    out: Optional[torch.Tensor] = None, p: Optional[int] = None,
-                   dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
+                   dev_status: Optional[torch.Tensor] = None, out_dtype: torch.dtype = torch.float32) -> torch.Tensor:
     """out[i] = SJLT_{k,s,seed}(g[i, idx]) for the rows of g (n x ld, fp32 or bf16).
     idx: uint32/int32 CUDA tensor of ascending coordinates, or None for the identity mask.
-    g may be a pinned host tensor: the kernel then reads the masked elements in place, across the bus."""
+    g may be a pinned host tensor: the kernel then reads the masked elements in place, across the bus.
+    The rows are written as fp32, or as bf16 (rounded once, at the final store) when `out` / `out_dtype` is bf16."""
     _need_device_readable(g)
     _need_cuda(idx, out, dev_status)
     _need_mask(idx)
@@ -206,12 +213,12 @@ def grass_compress(g: torch.Tensor, idx: Optional[torch.Tensor], k: int, s: int,
     p = g.shape[1] if p is None else p
     kprime = p if idx is None else idx.numel()
     if out is None:
-        out = torch.empty((n, k), dtype=torch.float32, device=_compute_device(g))
-    assert out.dtype == torch.float32 and out.stride(1) == 1
+        out = torch.empty((n, k), dtype=out_dtype, device=_compute_device(g))
+    assert out.dtype in (torch.float32, torch.bfloat16) and out.stride(1) == 1
     spec = SjltSpec(k, s, seed & 0xFFFFFFFFFFFFFFFF)
-    _check(lib().grass_compress(_ptr(g), _dt(g), n, p, ld, _ptr(idx), kprime, ctypes.byref(spec), _ptr(out),
-                                out.stride(0) if n > 1 else max(out.shape[1], k), _ptr(dev_status), _stream()),
-           "grass_compress")
+    _check(lib().grass_compress_out(_ptr(g), _dt(g), n, p, ld, _ptr(idx), kprime, ctypes.byref(spec), _ptr(out),
+                                    _dt(out), out.stride(0) if n > 1 else max(out.shape[1], k), _ptr(dev_status),
+                                    _stream()), "grass_compress")
     return out
 
 
@@ -312,13 +319,14 @@ def factgrass_grouped_workspace_bytes(L: int) -> int:
 
 def factgrass_compress_grouped(group: GroupedLayers, out: torch.Tensor, workspace: torch.Tensor,
                                dev_status: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """All layers of ``group`` in one launch; layer l fills out[:, off_l : off_l + k_l]."""
+    """All layers of ``group`` in one launch; layer l fills out[:, off_l : off_l + k_l].  `out` is fp32, or bf16
+    (every output rounded once, at the final store; see factgrass_compress_grouped_out in include/grass.h)."""
     _need_cuda(out, workspace, dev_status)
-    assert out.dtype == torch.float32 and out.stride(1) == 1
-    _check(lib().factgrass_compress_grouped(group.array, group.L, group.dtype, group.B, group.T, _ptr(out),
-                                            out.stride(0) if out.shape[0] > 1 else out.shape[1], _ptr(workspace),
-                                            workspace.numel() * workspace.element_size(), _ptr(dev_status),
-                                            _stream()), "factgrass_compress_grouped")
+    assert out.dtype in (torch.float32, torch.bfloat16) and out.stride(1) == 1
+    _check(lib().factgrass_compress_grouped_out(group.array, group.L, group.dtype, group.B, group.T, _ptr(out),
+                                                _dt(out), out.stride(0) if out.shape[0] > 1 else out.shape[1],
+                                                _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                                _ptr(dev_status), _stream()), "factgrass_compress_grouped")
     return out
 
 

@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(kFgThreads)
 factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ LayerDesc single, int32_t B,
                  int32_t T, const int64_t* __restrict__ tok_begin, const int32_t* __restrict__ tok_count,
                  int32_t max_tiles, int32_t chunk_len, float* __restrict__ out, int64_t ld_out,
-                 uint32_t* dev_status, int nprod)
+                 uint32_t* dev_status, int nprod, int flush_mode)
 {
     using elem_t = typename in_elem<F32>::type;
     constexpr int NP = F32 ? 3 : 1;                       // bf16 pieces per operand
@@ -289,7 +289,12 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
         __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(ACC_COLS) : "memory");
     }
-    if (smem_bins && ok) {
+    // flush_mode 0: several thread blocks feed the row: reductions into the zeroed row.  1 / 2: this thread block is
+    // the only one of its (layer, sample), so the bins ARE the row: plain stores, fp32 or bf16 (rounded here, once)
+    if (smem_bins && flush_mode != 0) {
+        for (uint32_t i = tid; i < k; i += kFgThreads)
+            store_out(out, (int64_t)b * ld_out + L.out_offset + i, bins[i], flush_mode == 2);
+    } else if (smem_bins && ok) {
         for (uint32_t i = tid; i < k; i += kFgThreads) {
             const float v = bins[i];
             if (v != 0.0f) atomicAdd(orow + i, v);
@@ -299,11 +304,12 @@ factgrass_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ La
 
 // zeroes every layer's [out_offset, out_offset + k) range of every sample row
 __global__ void factgrass_zero_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ LayerDesc single,
-                                      float* __restrict__ out, int64_t ld_out)
+                                      float* __restrict__ out, int64_t ld_out, int out_bf16)
 {
     const LayerDesc& L = descs ? descs[blockIdx.z] : single;
-    float* orow = out + (int64_t)blockIdx.y * ld_out + L.out_offset;
-    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < L.k; i += gridDim.x * blockDim.x) orow[i] = 0.0f;
+    const int64_t orow = (int64_t)blockIdx.y * ld_out + L.out_offset;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < L.k; i += gridDim.x * blockDim.x)
+        store_out(out, orow + i, 0.0f, out_bf16);
 }
 
 static grass_status fill_desc(LayerDesc& d, const factgrass_layer& l, int tile, int32_t T)
@@ -338,7 +344,7 @@ static grass_status fill_desc(LayerDesc& d, const factgrass_layer& l, int tile, 
 static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, grass_dtype dt, int32_t B, int32_t T,
                                   const int64_t* tok_begin, const int32_t* tok_count, float* out, int64_t ld_out,
                                   void* workspace, size_t workspace_bytes, uint32_t* dev_status, cudaStream_t st,
-                                  int epi = kEpiSjlt)
+                                  int epi = kEpiSjlt, int out_bf16 = 0)
 {
     if (L < 0 || B < 0 || T < 0 || (L > 0 && !layers)) return GRASS_ERR_INVALID_ARG;
     if (dt != GRASS_BF16 && dt != GRASS_F32) return GRASS_ERR_INVALID_ARG;
@@ -364,6 +370,12 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     if (!workspace && L != 1) return GRASS_ERR_INVALID_ARG;
     if (workspace && (workspace_bytes < (size_t)L * sizeof(LayerDesc) || ((uintptr_t)workspace & 15)))
         return GRASS_ERR_INVALID_ARG;
+    // every layer is checked on the host before anything touches the device
+    for (int l = 0; l < L; ++l) {
+        LayerDesc probe;
+        const grass_status rc = fill_desc(probe, layers[l], tile, T);
+        if (rc != GRASS_OK) return rc;
+    }
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
@@ -428,13 +440,16 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
     }
     if (cluster_nc > 0)
         return launch_factgrass_cluster(dev_descs, single, cplan, L, B, T, tok_begin, tok_count, cluster_nc,
-                                        cluster_chunk, out, ld_out, dev_status, st);
+                                        cluster_chunk, out, ld_out, dev_status, st, out_bf16);
+    // A bf16 row is rounded once, at the final store, so the streaming kernel takes it only where one thread block
+    // owns a whole (layer, sample): one block tile, the whole token sum (at most 8,192 tokens), bins in shared memory
+    if (out_bf16 && (max_tiles > 1 || max_k != max_k_smem || T > 8192 || epi != kEpiSjlt)) return GRASS_ERR_UNSUPPORTED;
 
     // zero the output ranges (the compress kernel accumulates partial projections into them)
     {
         dim3 zg((max_k + 1023) / 1024 > 0 ? (max_k + 1023) / 1024 : 1, (unsigned)B, (unsigned)L);
         if (zg.x > 64) zg.x = 64;
-        factgrass_zero_kernel<<<zg, 256, 0, st>>>(dev_descs, single, out, ld_out);
+        factgrass_zero_kernel<<<zg, 256, 0, st>>>(dev_descs, single, out, ld_out, out_bf16);
         if (launch_status() != GRASS_OK) return GRASS_ERR_CUDA;
     }
     if (T == 0 || max_tiles == 0) return GRASS_OK;
@@ -491,6 +506,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
         int chunk_len = (int)((T + want - 1) / want);
         chunk_len = (chunk_len + kTokTile - 1) / kTokTile * kTokTile;
         chunk_len = (int)tuning(GRASS_TUNE_FACTGRASS_CHUNK, chunk_len);
+        if (out_bf16) chunk_len = T;
         if (chunk_len < kTokTile) chunk_len = kTokTile;
         chunk_len = (chunk_len + kTokTile - 1) / kTokTile * kTokTile;
         const int nchunks = (T + chunk_len - 1) / chunk_len;
@@ -498,7 +514,7 @@ static grass_status run_factgrass(const factgrass_layer* layers, int32_t L, gras
         int nprod = (int)tuning(GRASS_TUNE_SPLIT_PRODUCTS, tc::kSplitProductsDefault);
         if (nprod != 3 && nprod != 4) nprod = 6;
         kern<<<grid, kFgThreads, smem, st>>>(dev_descs, single, B, T, tok_begin, tok_count, max_tiles, chunk_len, out,
-                                             ld_out, dev_status, nprod);
+                                             ld_out, dev_status, nprod, out_bf16 ? 2 : 0);
         return launch_status();
     };
     const size_t piece = (size_t)tile * tc::ROW_BYTES * 2;   // one bf16 piece of the A tile plus one of the G tile
@@ -575,7 +591,7 @@ grass_status launch_fim(const float* X, int64_t n, int64_t k, int64_t ld, float 
     int nprod = (int)tuning(GRASS_TUNE_SPLIT_PRODUCTS, tc::kSplitProductsDefault);
     if (nprod != 3 && nprod != 4) nprod = 6;
     kern<<<grid, kFgThreads, smem, st>>>(nullptr, d, 1, (int32_t)n, nullptr, nullptr, d.tiles_m * d.tiles_n,
-                                         (int32_t)chunk_len, F, ld_f, nullptr, nprod);
+                                         (int32_t)chunk_len, F, ld_f, nullptr, nprod, 0);
     return launch_status();
 }
 
@@ -667,6 +683,17 @@ extern "C" grass_status factgrass_compress_grouped(const factgrass_layer* layers
     if (!workspace) return GRASS_ERR_INVALID_ARG;
     return grass::run_factgrass(layers, L, dt, B, T, nullptr, nullptr, out, ld_out, workspace, workspace_bytes,
                                 dev_status, (cudaStream_t)stream);
+}
+
+extern "C" grass_status factgrass_compress_grouped_out(const factgrass_layer* layers, int32_t L, grass_dtype dt,
+                                                       int32_t B, int32_t T, void* out, grass_dtype out_dt,
+                                                       int64_t ld_out, void* workspace, size_t workspace_bytes,
+                                                       uint32_t* dev_status, void* stream)
+{
+    if (out_dt != GRASS_F32 && out_dt != GRASS_BF16) return GRASS_ERR_UNSUPPORTED;
+    if (!workspace && L > 1) return GRASS_ERR_INVALID_ARG;
+    return grass::run_factgrass(layers, L, dt, B, T, nullptr, nullptr, (float*)out, ld_out, workspace, workspace_bytes,
+                                dev_status, (cudaStream_t)stream, grass::kEpiSjlt, out_dt == GRASS_BF16);
 }
 
 extern "C" grass_status factgrass_compress_grouped_varlen(const factgrass_layer* layers, int32_t L, grass_dtype dt,

@@ -102,7 +102,8 @@ template <int TM, int TN>
 __global__ void __launch_bounds__(kFgThreads, 1)
 factgrass_cluster_kernel(const LayerDesc* __restrict__ descs, const __grid_constant__ LayerDesc single, int32_t T,
                          const int64_t* __restrict__ tok_begin, const int32_t* __restrict__ tok_count,
-                         int32_t chunk_len, float* __restrict__ out, int64_t ld_out, uint32_t* dev_status)
+                         int32_t chunk_len, float* __restrict__ out, int64_t ld_out, uint32_t* dev_status,
+                         int out_bf16)
 {
     static_assert((TM == 64 && TN == 64) || (TM == 128 && TN == 128), "tile");
     constexpr int A_TILE = TM * (int)tc::ROW_BYTES, G_TILE = TN * (int)tc::ROW_BYTES;
@@ -328,12 +329,12 @@ factgrass_cluster_kernel(const LayerDesc* __restrict__ descs, const __grid_const
     }
     cluster.sync();      // ... and after this barrier nobody touches another thread block's memory
     if (nc_ok) {
-        float* orow = out + (int64_t)b * ld_out + L.out_offset;
+        const int64_t orow = (int64_t)b * ld_out + L.out_offset;
         const uint32_t lo = rank * per, hi = min(lo + per, k);
         for (uint32_t i = lo + tid; i < hi; i += kFgThreads) {
             float acc = 0.0f;
             for (uint32_t q = 0; q < nc; ++q) acc += recv_bins[q * per + (i - lo)];
-            orow[i] = acc;
+            store_out(out, orow + i, acc, out_bf16);
         }
     }
 }
@@ -375,7 +376,7 @@ bool cluster_path_fits(const LayerDesc* d, int32_t L, ClusterPlan* plan)
 grass_status launch_factgrass_cluster(const LayerDesc* dev_descs, const LayerDesc& single, const ClusterPlan& plan,
                                       int32_t L, int32_t B, int32_t T, const int64_t* tok_begin,
                                       const int32_t* tok_count, int32_t nc, int32_t chunk_len, float* out,
-                                      int64_t ld_out, uint32_t* dev_status, cudaStream_t st)
+                                      int64_t ld_out, uint32_t* dev_status, cudaStream_t st, int out_bf16)
 {
     auto launch = [&](auto kern) -> grass_status {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem) != cudaSuccess)
@@ -403,7 +404,7 @@ grass_status launch_factgrass_cluster(const LayerDesc* dev_descs, const LayerDes
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         cudaError_t e = cudaLaunchKernelEx(&cfg, kern, dev_descs, single, T, tok_begin, tok_count, chunk_len, out,
-                                           ld_out, dev_status);
+                                           ld_out, dev_status, out_bf16);
         return e == cudaSuccess ? launch_status() : GRASS_ERR_CUDA;
     };
     if (plan.tile_m == 64) return launch(factgrass_cluster_kernel<64, 64>);

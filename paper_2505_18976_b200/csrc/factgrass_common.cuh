@@ -55,6 +55,6 @@ bool cluster_path_fits(const LayerDesc* host_descs, int32_t L, ClusterPlan* plan
 grass_status launch_factgrass_cluster(const LayerDesc* dev_descs, const LayerDesc& single, const ClusterPlan& plan,
                                       int32_t L, int32_t B, int32_t T, const int64_t* tok_begin,
                                       const int32_t* tok_count, int32_t nc, int32_t chunk_len, float* out,
-                                      int64_t ld_out, uint32_t* dev_status, cudaStream_t st);
+                                      int64_t ld_out, uint32_t* dev_status, cudaStream_t st, int out_bf16);
 
 }  // namespace grass

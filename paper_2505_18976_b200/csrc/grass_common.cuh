@@ -68,6 +68,14 @@ __device__ __forceinline__ uint16_t gather_u16(const uint16_t* p)
 __device__ __forceinline__ float elem_value(float x) { return x; }
 __device__ __forceinline__ float elem_value(__nv_bfloat16 x) { return __bfloat162float(x); }
 
+// final store of a compressed value: fp32, or bf16 rounded to nearest even (a cache of compressed vectors kept
+// at half the size; everything before the store is fp32)
+__device__ __forceinline__ void store_out(float* out, int64_t off, float v, int out_bf16)
+{
+    if (out_bf16) reinterpret_cast<__nv_bfloat16*>(out)[off] = __float2bfloat16_rn(v);
+    else out[off] = v;
+}
+
 template <typename T> struct elem;
 template <> struct elem<float> {
     static __device__ __forceinline__ float load(const float* p)
@@ -88,7 +96,7 @@ bool compress_rows_fits(const void* g, size_t elem_bytes, int64_t p, int64_t ld,
                         uint32_t k, int64_t n);
 grass_status launch_compress_rows(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld, const uint32_t* idx,
                                   int64_t kprime, const grass_sjlt_spec& sp, float* out, int64_t ld_out,
-                                  uint32_t* dev_status, cudaStream_t st);
+                                  uint32_t* dev_status, cudaStream_t st, int out_bf16);
 
 // launch-shape override set through grass_set_tuning, or `dflt` while the key is on automatic
 int64_t tuning(grass_tuning_key key, int64_t dflt);

@@ -48,7 +48,7 @@ __global__ void __launch_bounds__(NT, DENSE ? 4 : (U >= 16 ? 1024 : 2048) / NT)
 grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
                       const uint32_t* __restrict__ idx, int64_t kprime, uint32_t k, uint32_t s,
                       uint64_t seed, float scale, float* __restrict__ out, int64_t ld_out,
-                      int64_t j_per_cta, int accumulate, int use_smem, uint32_t* dev_status)
+                      int64_t j_per_cta, int accumulate, int use_smem, uint32_t* dev_status, int out_bf16)
 {
     extern __shared__ float bins[];  // S * k when use_smem
     const int tid = threadIdx.x;
@@ -267,11 +267,10 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
         const uint32_t per = (k + nr - 1) / nr;
         const uint32_t lo = r * per, hi = (lo + per) < k ? (lo + per) : k;
         for (int si = 0; si < ns; ++si) {
-            float* dst = out + (i0 + si) * ld_out;
             for (uint32_t i = lo + tid; i < hi; i += nthr) {
                 float acc = 0.0f;
                 for (uint32_t q = 0; q < nr; ++q) acc += cluster.map_shared_rank(bins, q)[(uint32_t)si * k + i];
-                dst[i] = acc;
+                store_out(out, (i0 + si) * ld_out + i, acc, out_bf16);
             }
         }
         cluster.sync();  // nobody leaves while its bins may still be read
@@ -286,7 +285,7 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
                     if (x != 0.0f) atomicAdd(dst + i, x);
                 }
             } else {
-                for (uint32_t i = tid; i < k; i += nthr) dst[i] = src[i];
+                for (uint32_t i = tid; i < k; i += nthr) store_out(out, (i0 + si) * ld_out + i, src[i], out_bf16);
             }
         }
     }
@@ -317,6 +316,7 @@ struct CompressPlan {
     int jsplit;     // CTAs that share one sample group (split of the masked positions)
     int use_smem;   // k-bin accumulators fit in shared memory
     int cluster;    // the jsplit CTAs are one thread-block cluster (DSMEM reduction)
+    int out_bf16;   // rows are stored as bf16 (final store only)
     int threads;    // threads per CTA of the gather path (256 or 512)
     int U;          // gathered loads in flight per thread and sample
 };
@@ -400,7 +400,7 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
         }
         const int use_smem = pl.use_smem;
         cudaError_t e = cudaLaunchKernelEx(&cfg, kern, g, n, p, ld, idx, kprime, sp.k, sp.s, sp.seed, scale, out,
-                                           ld_out, j_per_cta, accumulate, use_smem, dev_status);
+                                           ld_out, j_per_cta, accumulate, use_smem, dev_status, pl.out_bf16);
         return e == cudaSuccess ? launch_status() : GRASS_ERR_CUDA;
     };
     if (pl.dense) {
@@ -418,14 +418,22 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
 template <typename T>
 static grass_status dispatch_compress(const T* g, int64_t n, int64_t p, int64_t ld, const uint32_t* idx,
                                       int64_t kprime, const grass_sjlt_spec& sp, float* out, int64_t ld_out,
-                                      uint32_t* dev_status, cudaStream_t st)
+                                      uint32_t* dev_status, cudaStream_t st, int out_bf16)
 {
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) != cudaSuccess) return GRASS_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GRASS_ERR_CUDA;
     const bool dense = idx == nullptr && tuning(GRASS_TUNE_COMPRESS_DENSE, 1) != 0 &&
                        (uintptr_t)g % (4 * sizeof(T)) == 0 && ld % 4 == 0;
-    const CompressPlan pl = plan_compress(n, kprime, sp.k, sms, dense);
+    CompressPlan pl = plan_compress(n, kprime, sp.k, sms, dense);
+    pl.out_bf16 = out_bf16;
+    if (out_bf16 && !pl.cluster && (pl.jsplit > 1 || !pl.use_smem)) {
+        // a bf16 row is rounded once, at the final store, so it needs a launch shape in which one thread block
+        // or one cluster owns the row: no partial sums in global memory
+        if (!pl.use_smem) return GRASS_ERR_UNSUPPORTED;
+        pl.jsplit = pl.jsplit > 8 ? 8 : pl.jsplit;
+        pl.cluster = pl.jsplit > 1;
+    }
     if (!pl.cluster && (pl.jsplit > 1 || !pl.use_smem)) {
         cudaError_t e = cudaMemset2DAsync(out, (size_t)ld_out * sizeof(float), 0, (size_t)sp.k * sizeof(float),
                                           (size_t)n, st);
@@ -463,21 +471,25 @@ extern "C" grass_status grass_mask(const void* g, grass_dtype dt, int64_t n, int
     return grass::launch_status();
 }
 
-extern "C" grass_status grass_compress(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld,
-                                       const uint32_t* idx, int64_t kprime, const grass_sjlt_spec* spec,
-                                       float* out, int64_t ld_out, uint32_t* dev_status, void* stream)
+extern "C" grass_status grass_compress_out(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld,
+                                           const uint32_t* idx, int64_t kprime, const grass_sjlt_spec* spec,
+                                           void* out_v, grass_dtype out_dt, int64_t ld_out, uint32_t* dev_status,
+                                           void* stream)
 {
     if (!spec || spec->k == 0 || spec->s == 0) return GRASS_ERR_INVALID_ARG;
     if (n < 0 || p < 0 || kprime < 0 || kprime > p || ld < p || ld_out < (int64_t)spec->k) return GRASS_ERR_INVALID_ARG;
     if (p >= 0xFFFFFFFFLL) return GRASS_ERR_INVALID_ARG;
     if (!idx && kprime != p && kprime != 0) return GRASS_ERR_INVALID_ARG;
     if (dt != GRASS_F32 && dt != GRASS_BF16) return GRASS_ERR_UNSUPPORTED;
+    if (out_dt != GRASS_F32 && out_dt != GRASS_BF16) return GRASS_ERR_UNSUPPORTED;
     if (n == 0) return GRASS_OK;
-    if (!out || (!g && kprime > 0)) return GRASS_ERR_INVALID_ARG;
+    if (!out_v || (!g && kprime > 0)) return GRASS_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
+    const int out_bf16 = out_dt == GRASS_BF16;
+    const size_t osz = out_bf16 ? 2 : 4;
+    float* out = (float*)out_v;     // the kernels index it as fp32 or bf16 at the final store (store_out)
     if (kprime == 0) {
-        return grass::cuda_ok(cudaMemset2DAsync(out, (size_t)ld_out * sizeof(float), 0,
-                                                (size_t)spec->k * sizeof(float), (size_t)n, st));
+        return grass::cuda_ok(cudaMemset2DAsync(out, (size_t)ld_out * osz, 0, (size_t)spec->k * osz, (size_t)n, st));
     }
     // Row staging for dense masks (grass_compress_rows.cu): whole rows through shared memory, window by window,
     // the masked elements picked from there.  It is built and parity-tested but not chosen automatically: on B200
@@ -487,10 +499,17 @@ extern "C" grass_status grass_compress(const void* g, grass_dtype dt, int64_t n,
     // load of the launch in flight at once.  GRASS_TUNE_COMPRESS_ROWS = 1 selects it.
     if (grass::tuning(GRASS_TUNE_COMPRESS_ROWS, 0) == 1 &&
         grass::compress_rows_fits(g, dt == GRASS_F32 ? 4 : 2, p, ld, idx, kprime, spec->k, n))
-        return grass::launch_compress_rows(g, dt, n, p, ld, idx, kprime, *spec, out, ld_out, dev_status, st);
+        return grass::launch_compress_rows(g, dt, n, p, ld, idx, kprime, *spec, out, ld_out, dev_status, st, out_bf16);
     if (dt == GRASS_F32)
         return grass::dispatch_compress<float>((const float*)g, n, p, ld, idx, kprime, *spec, out, ld_out,
-                                               dev_status, st);
+                                               dev_status, st, out_bf16);
     return grass::dispatch_compress<__nv_bfloat16>((const __nv_bfloat16*)g, n, p, ld, idx, kprime, *spec, out,
-                                                   ld_out, dev_status, st);
+                                                   ld_out, dev_status, st, out_bf16);
+}
+
+extern "C" grass_status grass_compress(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld,
+                                       const uint32_t* idx, int64_t kprime, const grass_sjlt_spec* spec,
+                                       float* out, int64_t ld_out, uint32_t* dev_status, void* stream)
+{
+    return grass_compress_out(g, dt, n, p, ld, idx, kprime, spec, out, GRASS_F32, ld_out, dev_status, stream);
 }

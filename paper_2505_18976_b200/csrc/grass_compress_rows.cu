@@ -73,7 +73,8 @@ template <typename T, bool S1>
 __global__ void __launch_bounds__(kRowsThreads)
 grass_compress_rows_kernel(const T* __restrict__ g, int64_t p, int64_t ld, const uint32_t* __restrict__ idx,
                            int64_t kprime, uint32_t k, uint32_t s, uint64_t seed, float scale,
-                           float* __restrict__ out, int64_t ld_out, uint32_t idx_smem_bytes, uint32_t* dev_status)
+                           float* __restrict__ out, int64_t ld_out, uint32_t idx_smem_bytes, uint32_t* dev_status,
+                           int out_bf16)
 {
     constexpr int64_t WIN = kWinBytes / (int)sizeof(T);      // coordinates per window
     // [kWinBufs windows][index list][k bins][per-warp queues: value, position]
@@ -204,8 +205,7 @@ grass_compress_rows_kernel(const T* __restrict__ g, int64_t p, int64_t ld, const
         }
         __syncthreads();
     }
-    float* dst = out + i * ld_out;
-    for (uint32_t b = tid; b < k; b += kRowsThreads) dst[b] = bins[b];
+    for (uint32_t b = tid; b < k; b += kRowsThreads) store_out(out, i * ld_out + b, bins[b], out_bf16);
 }
 
 static size_t rows_smem_bytes(int64_t kprime, uint32_t k, uint32_t* idx_bytes)
@@ -229,7 +229,7 @@ bool compress_rows_fits(const void* g, size_t elem_bytes, int64_t p, int64_t ld,
 template <typename T>
 static grass_status launch_rows_t(const T* g, int64_t n, int64_t p, int64_t ld, const uint32_t* idx, int64_t kprime,
                                   const grass_sjlt_spec& sp, float* out, int64_t ld_out, uint32_t* dev_status,
-                                  cudaStream_t st)
+                                  cudaStream_t st, int out_bf16)
 {
     uint32_t idx_bytes = 0;
     const size_t smem = rows_smem_bytes(kprime, sp.k, &idx_bytes);
@@ -238,7 +238,7 @@ static grass_status launch_rows_t(const T* g, int64_t n, int64_t p, int64_t ld, 
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return GRASS_ERR_CUDA;
         kern<<<dim3((unsigned)n, 1, 1), kRowsThreads, smem, st>>>(g, p, ld, idx, kprime, sp.k, sp.s, sp.seed, scale, out,
-                                                                  ld_out, idx_bytes, dev_status);
+                                                                  ld_out, idx_bytes, dev_status, out_bf16);
         return launch_status();
     };
     if (sp.s == 1) return launch(grass_compress_rows_kernel<T, true>);
@@ -247,11 +247,12 @@ static grass_status launch_rows_t(const T* g, int64_t n, int64_t p, int64_t ld, 
 
 grass_status launch_compress_rows(const void* g, grass_dtype dt, int64_t n, int64_t p, int64_t ld, const uint32_t* idx,
                                   int64_t kprime, const grass_sjlt_spec& sp, float* out, int64_t ld_out,
-                                  uint32_t* dev_status, cudaStream_t st)
+                                  uint32_t* dev_status, cudaStream_t st, int out_bf16)
 {
     if (dt == GRASS_F32)
-        return launch_rows_t<float>((const float*)g, n, p, ld, idx, kprime, sp, out, ld_out, dev_status, st);
-    return launch_rows_t<__nv_bfloat16>((const __nv_bfloat16*)g, n, p, ld, idx, kprime, sp, out, ld_out, dev_status, st);
+        return launch_rows_t<float>((const float*)g, n, p, ld, idx, kprime, sp, out, ld_out, dev_status, st, out_bf16);
+    return launch_rows_t<__nv_bfloat16>((const __nv_bfloat16*)g, n, p, ld, idx, kprime, sp, out, ld_out, dev_status, st,
+                                        out_bf16);
 }
 
 }  // namespace grass
