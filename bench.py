@@ -200,8 +200,9 @@ class GrassJob:
 class FactJob:
     """configs 3-5: all layers through one factgrass_compress_grouped launch (+ score for config 5)."""
 
-    def __init__(self, cfg, device, G, W, seq_len_aware=False, fp32_inputs=False, precondition=False):
+    def __init__(self, cfg, device, G, W, seq_len_aware=False, fp32_inputs=False, precondition=False, out_bf16=False):
         self.cfg, self.G, self.device = cfg, G, device
+        self.out_bf16 = out_bf16
         self.fp32 = fp32_inputs
         eb = 4 if fp32_inputs else 2
         layers, alg, line = [], 0, 0
@@ -226,7 +227,7 @@ class FactJob:
             self.dense += cfg.B * cfg.T * (lay.d_in + lay.d_out) * eb
         self.layers = layers
         self.group = G.GroupedLayers(layers)
-        self.out = torch.empty((cfg.B, cfg.out_dim), dtype=torch.float32, device=device)
+        self.out = torch.empty((cfg.B, cfg.out_dim), dtype=torch.bfloat16 if out_bf16 else torch.float32, device=device)
         self.ws = torch.empty(G.factgrass_grouped_workspace_bytes(len(layers)), dtype=torch.uint8, device=device)
         self.score = None
         if cfg.score_n_train:
@@ -286,6 +287,8 @@ class FactJob:
             d["score"] = f"{c.score_n_train}x{c.score_n_test}x{c.k} fp32"
         if self.fp32:
             d["inputs"] = "fp32"
+        if self.out_bf16:
+            d["compressed_rows"] = "bf16 (rounded at the final store)"
         if self.precondition:
             d["score"] += ", preconditioned by the damped projected FIM (lambda 0.1)"
         if self.tok_count is not None:
@@ -308,11 +311,12 @@ def small_config(cfg_id, W):
     return cfg
 
 
-def make_job(cfg_id, device, G, W, small=False, seq_len_aware=False, fp32_inputs=False, precondition=False):
+def make_job(cfg_id, device, G, W, small=False, seq_len_aware=False, fp32_inputs=False, precondition=False,
+             out_bf16=False):
     cfg = small_config(cfg_id, W) if small else W.CONFIGS[cfg_id]
     if cfg_id in (1, 2):
         return GrassJob(cfg, device, G, W)
-    return FactJob(cfg, device, G, W, seq_len_aware, fp32_inputs, precondition)
+    return FactJob(cfg, device, G, W, seq_len_aware, fp32_inputs, precondition, out_bf16)
 
 
 def time_job(job, steps, warmup, world, device):
@@ -722,6 +726,11 @@ def main():
     ap.add_argument("--fp32-inputs", action="store_true", help="configs 3-5: fp32 A and G instead of bf16")
     ap.add_argument("--precondition", action="store_true",
                     help="config 5: projected FIM of the train vectors, damped solve for the test vectors, then scores")
+    ap.add_argument("--tune", action="append", default=[], metavar="KEY=VALUE",
+                    help="force a launch-shape choice of the library (grass_set_tuning), e.g. factgrass_path=0; "
+                         "for profiler captures and sweeps")
+    ap.add_argument("--out-bf16", action="store_true",
+                    help="configs 3-5: compressed rows written as bf16 by the compress call (not a bench line)")
     ap.add_argument("--seq-len-aware", action="store_true",
                     help="configs 3-5: pass per-sample token counts so that padding tokens are not read")
     args = ap.parse_args()
@@ -739,6 +748,9 @@ def main():
     device = torch.device("cuda", local)
     import paper_2505_18976_b200 as G
     G.lib()
+    for kv in args.tune:
+        key, val = kv.split("=")
+        G.grass_set_tuning(key, int(val))
     warmup = args.warmup if args.small else max(args.warmup, 3)
     if args.fig4:
         if rank == 0:
@@ -763,7 +775,7 @@ def main():
         ms_per_step, dom_ms, warm_ms, dirty_ms = time_job(job, steps, warmup, world, device)
         clocks = sampler.stop()
         achieved = job.alg_bytes_per_launch / (dom_ms * 1e-3) / 1e9
-        plain = not (kw.get("fp32_inputs") or kw.get("seq_len_aware") or kw.get("small"))
+        plain = not (kw.get("fp32_inputs") or kw.get("seq_len_aware") or kw.get("small") or kw.get("out_bf16"))
         roofline = {"bound": "hbm", "kernel": job.dominant, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "peak_source": peak_src,
                     "algorithmic_bytes_per_launch": int(job.alg_bytes_per_launch),
@@ -780,8 +792,8 @@ def main():
 
     job, ms_per_step, clocks, roofline, extra = measure(args.config, args.steps, small=args.small,
                                                         seq_len_aware=args.seq_len_aware, fp32_inputs=args.fp32_inputs,
-                                                        precondition=args.precondition)
-    if args.fp32_inputs or args.precondition:
+                                                        precondition=args.precondition, out_bf16=args.out_bf16)
+    if args.fp32_inputs or args.precondition or args.out_bf16:
         args.no_e2e = True      # the host-buffer leg covers the default path only
     value = world * job.samples_per_step / (ms_per_step * 1e-3)
 
@@ -796,7 +808,7 @@ def main():
     # fewer steps), so that one line carries all five; `value` stays the default workload's.
     per_config = None
     default_run = (args.config == 5 and not (args.small or args.fp32_inputs or args.precondition or args.seq_len_aware
-                                             or args.no_per_config))
+                                             or args.no_per_config or args.out_bf16 or args.tune))
     if default_run:
         main_desc = job.desc()
         kernels_main = job.kernels_per_step * args.steps
@@ -825,6 +837,8 @@ def main():
         cfgd.update(extra)
         if args.small:
             cfgd["small"] = True
+        if args.tune:
+            cfgd["tuning"] = args.tune
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
                 "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16" if (args.config >= 3 and not args.fp32_inputs) else "f32", "data": "synthetic", "config": cfgd,
@@ -841,8 +855,8 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel per launch, from ncu captures
 # summarised under profiles/ (bytes; None until captured)
-TRAFFIC = {1: 58_786_304 + 489_984, 2: 8 * (239_941_632 + 3_357_184), 3: 101_295_360 + 3_341_312,
-           4: 3 * (1_044_521_000 + 3_736_576), 5: 16 * (729_330_432 + 4_238_848)}
+TRAFFIC = {1: 58_790_400 + 459_008, 2: 8 * (239_980_032 + 3_712_256), 3: 100_758_016 + 3_166_464,
+           4: 3 * (1_044_538_368 + 3_582_976), 5: 16 * (729_330_944 + 4_280_320)}
 
 if __name__ == "__main__":
     main()
