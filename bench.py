@@ -677,11 +677,40 @@ def compare_compressors(cfg_id, device, G, W, steps=5):
                         "ms_per_batch": res, "tokens_per_s": {n: tokens / (ms * 1e-3) for n, ms in res.items()}}}
 
 
+def reference_full(args, W):
+    """--impl reference --full: the oracle over the WHOLE FactGraSS configuration, one step, layer by layer (the inputs
+    of a layer are drawn, untimed, just before its call, so the host never holds more than one layer)."""
+    import oracle
+    oracle.build()
+    cfg = W.CONFIGS[args.config]
+    total = 0.0
+    for l, lay in enumerate(cfg.layers):
+        A, Gt = W.layer_io(cfg, l, device="cpu")
+        s_in, s_out = W.layer_mask_seeds(cfg, l)
+        mi, mo = oracle.random_mask(lay.d_in, cfg.kin, s_in), oracle.random_mask(lay.d_out, cfg.kout, s_out)
+        a, g = W.bits_of(A), W.bits_of(Gt)
+        t0 = time.perf_counter()
+        oracle.factgrass(a, g, mi, mo, cfg.k, cfg.s, W.layer_hash_seed(cfg, l), want_absum=False)
+        total += time.perf_counter() - t0
+    cores = min(oracle.num_threads(), len(os.sched_getaffinity(0)))
+    what = f"all {len(cfg.layers)} layers, all {cfg.B} samples x {cfg.T} tokens, one step (the score step is not included)"
+    val = cfg.B / total
+    print(json.dumps({"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": 1,
+                      "warmup": 0, "ms_per_step": total * 1e3, "higher_is_better": True, "scaling": "weak",
+                      "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                      "config": {"workload": cfg.name, "sample": what},
+                      "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+                      "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                      "gpu_launches": 0}))
+
+
 def reference_arm(args, W):
     """--impl reference: the CPU oracle, as it stands, timed on the host cores."""
     world, rank, _ = int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), 0
     if rank != 0:
         return
+    if args.full and args.config >= 3:
+        return reference_full(args, W)
     import oracle
     oracle.build()
     run, sample_equiv, what = oracle_sample(args.config, W)
@@ -711,6 +740,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=5, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--full", action="store_true",
+                    help="with --impl reference, configs 3-5: the oracle over the whole configuration, one step "
+                         "(minutes; the default is a bounded sample)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-per-config", action="store_true",
