@@ -340,8 +340,18 @@ static CompressPlan plan_compress(int64_t n, int64_t kprime, uint32_t k, int sm_
     int U = S == 1 ? 8 : (S == 8 ? 2 : 4);
     if (S == 1 && !dense && tuning(GRASS_TUNE_COMPRESS_LOADS, 8) == 16) U = 16;
     pl.U = U;
-    pl.threads = (!dense && tuning(GRASS_TUNE_COMPRESS_THREADS, kThreads) == 2 * kThreads) ? 2 * kThreads : kThreads;
     const int64_t groups = (n + S - 1) / S;
+    pl.threads = kThreads;
+    if (!dense) {
+        // With a row for every SM, a thread block of up to 1,024 threads takes a whole row in one round of loads:
+        // no position split, so no cluster, no exchange of bins and no thread blocks left waiting for a slot
+        // (config 1: 25.2 -> 22.9 us).  Longer masks and fewer rows keep 256 threads and split the positions.
+        int t = kThreads;
+        if (S == 1 && groups >= sm_count && kprime <= (int64_t)4 * kThreads * U)
+            while ((int64_t)t * U < kprime) t *= 2;
+        t = (int)tuning(GRASS_TUNE_COMPRESS_THREADS, t);
+        if (t == 2 * kThreads || t == 4 * kThreads) pl.threads = t;
+    }
     // split positions until there are ~4 CTAs per SM, but keep one full round of loads per CTA
     const int64_t round = (int64_t)pl.threads * U;
     const int64_t max_js = kprime / round > 0 ? kprime / round : 1;
@@ -410,6 +420,10 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
     if (pl.threads == 2 * kThreads) {
         if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true, false, 2 * kThreads>);
         return launch(grass_compress_kernel<T, S, U, false, false, 2 * kThreads>);
+    }
+    if (pl.threads == 4 * kThreads) {
+        if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true, false, 4 * kThreads>);
+        return launch(grass_compress_kernel<T, S, U, false, false, 4 * kThreads>);
     }
     if (sp.s == 1) return launch(grass_compress_kernel<T, S, U, true, false, kThreads>);
     return launch(grass_compress_kernel<T, S, U, false, false, kThreads>);

@@ -172,6 +172,15 @@ def test_grass_compress_launch_shapes(G, W, oracle_mod, tune, S, js, cluster):
     _grass_case(G, W, oracle_mod, 5, 40_000, 9_000, 1_003, s=2)
 
 
+@pytest.mark.parametrize("threads,loads", [(512, 8), (1024, 8), (256, 16), (1024, 16)])
+def test_grass_compress_block_sizes(G, W, oracle_mod, tune, threads, loads):
+    """Thread blocks of 512 and 1,024 threads and 16 loads per thread: one round or several, ragged tails, s = 2."""
+    tune(compress_threads=threads, compress_loads=loads)
+    _grass_case(G, W, oracle_mod, 7, 40_000, 9_000, 1_000)
+    _grass_case(G, W, oracle_mod, 3, 70_000, 33_333, 257, s=2)
+    _grass_case(G, W, oracle_mod, 200, 20_000, 5_000, 300, dtype=torch.bfloat16)   # a row per SM: whole-row blocks
+
+
 def test_grass_compress_special_values(G, oracle_mod):
     """All-zero rows give exact zeros; NaN / Inf reach exactly the bins they hash to."""
     n, p, k, seed = 4, 5_000, 64, 3
