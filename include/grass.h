@@ -328,8 +328,9 @@ typedef enum {
     GRASS_TUNE_FACTGRASS_PATH = 10,    /* factgrass: 0 = streaming kernel, 1 = cluster kernel (see factgrass.cu) */
     GRASS_TUNE_COMPRESS_ROWS = 11,     /* grass_compress: 0 = never stage row segments in shared memory, 1 = wherever the operands allow */
     GRASS_TUNE_COMPRESS_LOADS = 12,    /* grass_compress gather path: loads in flight per thread (4, 8, 16) */
-    GRASS_TUNE_COMPRESS_THREADS = 13,  /* grass_compress gather path: threads per block (256, 512) */
-    GRASS_TUNE_COUNT = 14
+    GRASS_TUNE_COMPRESS_THREADS = 13,  /* grass_compress gather path: threads per block (256, 512, 1024) */
+    GRASS_TUNE_COMPRESS_IDX_SMEM = 14, /* grass_compress gather path: 0 = never copy the index list into shared memory */
+    GRASS_TUNE_COUNT = 15
 } grass_tuning_key;
 #define GRASS_TUNE_AUTO (-1)
 grass_status grass_set_tuning(grass_tuning_key key, int64_t value);

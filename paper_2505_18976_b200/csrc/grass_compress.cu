@@ -12,6 +12,7 @@
 // With the identity mask on vector-aligned rows (plain SJLT) the rows are streamed with 16-byte loads instead
 // of gathers.  grass_mask (Mask alone, Section 3.2) is the gather without the projection.
 #include "grass_common.cuh"
+#include "tcgen05_util.cuh"
 
 #include <cooperative_groups.h>
 
@@ -48,7 +49,8 @@ __global__ void __launch_bounds__(NT, DENSE ? 4 : (U >= 16 ? 1024 : 2048) / NT)
 grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
                       const uint32_t* __restrict__ idx, int64_t kprime, uint32_t k, uint32_t s,
                       uint64_t seed, float scale, float* __restrict__ out, int64_t ld_out,
-                      int64_t j_per_cta, int accumulate, int use_smem, uint32_t* dev_status, int out_bf16)
+                      int64_t j_per_cta, int accumulate, int use_smem, uint32_t* dev_status, int out_bf16,
+                      uint32_t idx_smem_bytes)
 {
     extern __shared__ float bins[];  // S * k when use_smem
     const int tid = threadIdx.x;
@@ -59,9 +61,33 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
     const int64_t j0 = (int64_t)blockIdx.y * j_per_cta;
     const int64_t j1 = (j0 + j_per_cta) < kprime ? (j0 + j_per_cta) : kprime;
 
-    if (use_smem) {
+    // Whole-row thread blocks keep the index list in shared memory (idx_smem_bytes > 0: one bulk copy, started
+    // before anything else): every thread block of the launch reads the whole list, and hundreds of them asking L2
+    // for the same few lines at once take microseconds to be served.
+    __shared__ __align__(8) unsigned long long idx_bar;
+    uint32_t* sidx = reinterpret_cast<uint32_t*>(bins + (use_smem ? ((size_t)S * k + 3) / 4 * 4 : 0));
+    const uint32_t idx_bulk = idx_smem_bytes ? (uint32_t)((kprime * 4) & ~(int64_t)15) : 0u;
+    if (idx_smem_bytes && tid == 0) {
+        const uint32_t bar = tc::smem_u32(&idx_bar);
+        tc::mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (idx_bulk > 0) {
+            tc::expect_tx(bar, idx_bulk);
+            tc::bulk_copy(tc::smem_u32(sidx), idx, idx_bulk, bar);
+        }
+    }
+    if (use_smem)
         for (uint32_t i = tid; i < (uint32_t)S * k; i += nthr) bins[i] = 0.0f;
-        __syncthreads();
+    if (idx_smem_bytes)
+        for (int64_t j = idx_bulk / 4 + tid; j < kprime; j += nthr) sidx[j] = __ldg(idx + j);   // at most 3 entries
+    if (use_smem || idx_smem_bytes) __syncthreads();
+    // the list has landed; should the bounded wait expire, the indices are read from global memory after all
+    // (after one more bounded wait: no copy may be in flight into shared memory that is about to be reused or left)
+    bool idx_in_smem = idx_smem_bytes != 0;
+    if (idx_bulk > 0 && !tc::mbar_wait(tc::smem_u32(&idx_bar), 0)) {
+        idx_in_smem = false;
+        if (tid == 0 && dev_status) atomicOr(dev_status, GRASS_DEV_TIMEOUT);
+        tc::mbar_wait(tc::smem_u32(&idx_bar), 0);
     }
 
     const T* rows[S];
@@ -192,7 +218,7 @@ grass_compress_kernel(const T* __restrict__ g, int64_t n, int64_t p, int64_t ld,
             const int64_t j = jb + (int64_t)u * nthr;
             ok[u] = j < j1;
             uint32_t c = 0;
-            if (ok[u]) c = idx ? __ldg(idx + j) : (uint32_t)j;
+            if (ok[u]) c = idx_in_smem ? sidx[j] : (idx ? __ldg(idx + j) : (uint32_t)j);
             if ((int64_t)c >= p) { bad = bad || ok[u]; ok[u] = false; c = 0; }
             col[u] = c;
         }
@@ -317,6 +343,7 @@ struct CompressPlan {
     int use_smem;   // k-bin accumulators fit in shared memory
     int cluster;    // the jsplit CTAs are one thread-block cluster (DSMEM reduction)
     int out_bf16;   // rows are stored as bf16 (final store only)
+    uint32_t idx_smem;  // bytes of shared memory for a copy of the index list (0: indices are read from global memory)
     int threads;    // threads per CTA of the gather path (256 or 512)
     int U;          // gathered loads in flight per thread and sample
 };
@@ -388,6 +415,7 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
     const int accumulate = pl.cluster ? 2 : ((pl.jsplit > 1 || !pl.use_smem) ? 1 : 0);
     size_t smem = pl.use_smem ? (size_t)S * sp.k * sizeof(float) : 0;
     if (pl.dense) smem = ((smem + 7) & ~(size_t)7) + kQueueBytes;      // the warps' non-zero queues
+    if (pl.idx_smem) smem = (smem + 15) / 16 * 16 + pl.idx_smem;       // a copy of the index list
     const float scale = 1.0f / sqrtf((float)sp.s);
     auto launch = [&](auto kern) -> grass_status {
         if (smem > 48 * 1024) {
@@ -410,7 +438,7 @@ static grass_status launch_compress(const T* g, int64_t n, int64_t p, int64_t ld
         }
         const int use_smem = pl.use_smem;
         cudaError_t e = cudaLaunchKernelEx(&cfg, kern, g, n, p, ld, idx, kprime, sp.k, sp.s, sp.seed, scale, out,
-                                           ld_out, j_per_cta, accumulate, use_smem, dev_status, pl.out_bf16);
+                                           ld_out, j_per_cta, accumulate, use_smem, dev_status, pl.out_bf16, pl.idx_smem);
         return e == cudaSuccess ? launch_status() : GRASS_ERR_CUDA;
     };
     if (pl.dense) {
@@ -441,6 +469,11 @@ static grass_status dispatch_compress(const T* g, int64_t n, int64_t p, int64_t 
                        (uintptr_t)g % (4 * sizeof(T)) == 0 && ld % 4 == 0;
     CompressPlan pl = plan_compress(n, kprime, sp.k, sms, dense);
     pl.out_bf16 = out_bf16;
+    // whole-row thread blocks, one for every SM or more: the index list (up to 48 KB) goes into shared memory
+    pl.idx_smem = 0;
+    if (!dense && idx && pl.jsplit == 1 && pl.S == 1 && pl.use_smem && n >= sms && kprime * 4 <= 48 * 1024 &&
+        (uintptr_t)idx % 16 == 0 && tuning(GRASS_TUNE_COMPRESS_IDX_SMEM, 1) != 0)
+        pl.idx_smem = (uint32_t)((kprime * 4 + 15) / 16 * 16);
     if (out_bf16 && !pl.cluster && (pl.jsplit > 1 || !pl.use_smem)) {
         // a bf16 row is rounded once, at the final store, so it needs a launch shape in which one thread block
         // or one cluster owns the row: no partial sums in global memory

@@ -58,16 +58,8 @@ __device__ __forceinline__ int64_t warp_lower_bound(const uint32_t* idx, int64_t
     return lo + __popc(__ballot_sync(0xFFFFFFFFu, below));
 }
 
-__device__ __forceinline__ void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ void expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
+using tc::bulk_copy;
+using tc::expect_tx;
 
 template <typename T, bool S1>
 __global__ void __launch_bounds__(kRowsThreads)

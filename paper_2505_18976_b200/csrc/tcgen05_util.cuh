@@ -53,6 +53,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     return false;
 }
 
+// untiled bulk copy global -> this thread block's shared memory; both addresses 16-byte aligned, `bytes` a multiple
+// of 16; completion is counted in bytes on the mbarrier
+__device__ __forceinline__ void bulk_copy(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
 // shared-memory matrix descriptor: K-major, 64-byte swizzle, version 1 (sm_100).  The leading-dimension
 // offset is not used by swizzled K-major layouts (set to 16 bytes).  A descriptor that starts 32 bytes
 // into the tile addresses k-values 16..31.
