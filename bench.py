@@ -887,7 +887,7 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel per launch, from ncu captures
 # summarised under profiles/ (bytes; None until captured)
-TRAFFIC = {1: 58_790_400 + 459_008, 2: 8 * (239_980_032 + 3_712_256), 3: 100_758_016 + 3_166_464,
+TRAFFIC = {1: 58_796_800 + 536_832, 2: 8 * (239_980_032 + 3_712_256), 3: 100_758_016 + 3_166_464,
            4: 3 * (1_044_538_368 + 3_582_976), 5: 16 * (729_330_944 + 4_280_320)}
 
 if __name__ == "__main__":
