@@ -330,7 +330,8 @@ typedef enum {
     GRASS_TUNE_COMPRESS_LOADS = 12,    /* grass_compress gather path: loads in flight per thread (4, 8, 16) */
     GRASS_TUNE_COMPRESS_THREADS = 13,  /* grass_compress gather path: threads per block (256, 512, 1024) */
     GRASS_TUNE_COMPRESS_IDX_SMEM = 14, /* grass_compress gather path: 0 = never copy the index list into shared memory */
-    GRASS_TUNE_COUNT = 15
+    GRASS_TUNE_SCORE_BF16_SOLO = 15,   /* grass_score_bf16: 0 = always thread-block pairs, also for M <= 256 */
+    GRASS_TUNE_COUNT = 16
 } grass_tuning_key;
 #define GRASS_TUNE_AUTO (-1)
 grass_status grass_set_tuning(grass_tuning_key key, int64_t value);

@@ -35,7 +35,7 @@ EXPORTS = ("grass_compress", "factgrass_compress", "factgrass_compress_grouped",
 TUNE = {"compress_samples": 0, "compress_jsplit": 1, "compress_cluster": 2, "compress_dense": 3,
         "factgrass_tile": 4, "factgrass_chunk": 5, "factgrass_carveout": 6, "score_ffma": 7, "score_splits": 8,
         "split_products": 9, "factgrass_path": 10, "compress_rows": 11, "compress_loads": 12,
-        "compress_threads": 13, "compress_idx_smem": 14}
+        "compress_threads": 13, "compress_idx_smem": 14, "score_bf16_solo": 15}
 
 
 class GrassError(RuntimeError):

@@ -572,6 +572,166 @@ grass_score_bf16_kernel(const __grid_constant__ CUtensorMap map_train, const __g
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// bf16 scores with one thread block per 128 x (<= 256) output tile (tcgen05.mma.cta_group::1): for a test set that
+// fits one column tile (M <= 256, the usual attribute-stage shape) the pair kernel above gains nothing from sharing
+// the test tile between two SMs and pays a remote barrier arrival per stage.  Here every thread block brings in its
+// own 128 train rows and ALL test rows of a k tile (the test rows come from L2 after the first block has read
+// them), one warp issues the loads, one thread the MMAs, four warps drain the accumulator; all barriers are local.
+constexpr int S_STAGES = 4;
+constexpr int S_A_BYTES = BM * H_ROW_BYTES;              // 128 train rows x 64 k-values: 16 KB
+constexpr int S_B_BYTES = BN * H_ROW_BYTES;              // up to 256 test rows x 64 k-values: 32 KB
+constexpr int S_STAGE_BYTES = S_A_BYTES + S_B_BYTES;
+constexpr int S_THREADS = (H_EPI_WARPS + 2) * 32;        // + MMA / tensor-memory warp, TMA warp
+static_assert(S_STAGES * S_STAGE_BYTES <= 224 * 1024 && S_STAGE_BYTES % 1024 == 0, "shared memory");
+
+__global__ void __launch_bounds__(S_THREADS, 1)
+grass_score_bf16_solo_kernel(const __grid_constant__ CUtensorMap map_train, const __grid_constant__ CUtensorMap map_test,
+                             int64_t N, int64_t M, int64_t D, int64_t kt_split, float* __restrict__ scores,
+                             int64_t ld_s, int out_vec_ok)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long bars[2 * S_STAGES + 1];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ volatile int abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t n0 = (int64_t)blockIdx.x * BM;
+    const int64_t m0 = (int64_t)blockIdx.y * BN;
+    const int64_t m_rows = (M - m0) < BN ? (M - m0) : BN;
+    const uint32_t n_mma = (uint32_t)((m_rows + 15) / 16 * 16);    // MMA N (a multiple of 16 for M = 128)
+    const int b_boxes = n_mma > (uint32_t)H_BOX_ROWS ? 2 : 1;      // boxes of 128 test rows per stage
+    const int64_t kt0 = (int64_t)blockIdx.z * kt_split;
+    const int64_t kt_left = (D + H_BK - 1) / H_BK - kt0;
+    const int64_t ktiles = kt_left < kt_split ? (kt_left > 0 ? kt_left : 0) : kt_split;
+    const bool add_out = gridDim.z > 1;
+
+    // full[s]: the tiles of stage s have landed; empty[s]: the MMAs that read stage s are done; accum: all MMAs are
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[S_STAGES]), accum = smem_u32(&bars[2 * S_STAGES]);
+    if (tid == 0) {
+        for (int s = 0; s < S_STAGES; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(accum, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == H_EPI_WARPS) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                     "r"(H_TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = tmem_base_slot;
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (warp < H_EPI_WARPS) {
+        // ---------------- epilogue: the 128 rows of the accumulator ----------------
+        bool ok = true;
+        if (ktiles > 0) ok = mbar_wait(accum, 0) && !abort_flag;
+        if (!ok) abort_flag = 1;
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int64_t row = n0 + warp * 32 + lane;
+        for (uint32_t c0 = 0; c0 < n_mma; c0 += 32) {
+            uint32_t v[32];
+            if (ok && ktiles > 0) {
+                tmem_ld32(tmem_d + ((uint32_t)(warp * 32) << 16) + c0, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[e] = (ktiles > 0) ? 0x7FC00000u : 0u;   // NaN marks an aborted tile
+            }
+            if (row < N) {
+                float* dst = scores + row * ld_s + m0 + c0;
+                const bool vec = out_vec_ok && (int64_t)(c0 + 32) <= m_rows;
+                if (add_out) {
+                    if (vec) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + e),
+                                         "f"(__uint_as_float(v[e])), "f"(__uint_as_float(v[e + 1])),
+                                         "f"(__uint_as_float(v[e + 2])), "f"(__uint_as_float(v[e + 3]))
+                                         : "memory");
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if ((int64_t)(c0 + e) < m_rows) atomicAdd(dst + e, __uint_as_float(v[e]));
+                    }
+                } else if (vec) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4)
+                        *reinterpret_cast<uint4*>(dst + e) = make_uint4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if ((int64_t)(c0 + e) < m_rows) dst[e] = __uint_as_float(v[e]);
+                }
+            }
+        }
+    } else if (warp == H_EPI_WARPS + 1) {
+        // ---------------- TMA: bf16 tiles straight into the operand stages (one thread) ----------------
+        if (lane == 0) {
+            const uint32_t stage_tx = (uint32_t)(S_A_BYTES + b_boxes * H_BOX_ROWS * H_ROW_BYTES);
+            const int64_t rot = (ktiles > 0 && ktiles <= 128) ? ((int64_t)blockIdx.x * ktiles / gridDim.x) % ktiles : 0;
+            int64_t issued = 0;
+            bool ok = true;
+            for (int64_t kt = 0; kt < ktiles; ++kt) {
+                const int s = (int)(kt % S_STAGES);
+                const uint32_t round = (uint32_t)(kt / S_STAGES);
+                if (round > 0) ok = mbar_wait(empty0 + 8 * s, (round - 1) & 1) && !abort_flag;
+                if (!ok) break;
+                mbar_expect_tx(full0 + 8 * s, stage_tx);
+                const uint32_t dst = smem_base + s * S_STAGE_BYTES;
+                // thread blocks walk the k tiles in rotated order (spread evenly over the contraction), so that at
+                // any moment they ask L2 for different tiles of the test matrix instead of all for the same one:
+                // 65 -> 56 us at 16,384 x 256 x 4,096; for long contractions it measured slower (143 -> 151 us at
+                // D = 16,384) and is left out
+                const int32_t x = (int32_t)((kt0 + (kt + rot) % ktiles) * H_BK);
+                tma_load_2d(dst, &map_train, x, (int32_t)n0, full0 + 8 * s);
+                for (int bx = 0; bx < b_boxes; ++bx)
+                    tma_load_2d(dst + S_A_BYTES + bx * H_BOX_ROWS * H_ROW_BYTES, &map_test, x,
+                                (int32_t)m0 + bx * H_BOX_ROWS, full0 + 8 * s);
+                issued = kt + 1;
+            }
+            if (!ok) abort_flag = 1;
+            // no copy of this thread block may still be in flight when it leaves
+            for (int64_t kt = issued > S_STAGES ? issued - S_STAGES : 0; kt < issued; ++kt)
+                if (!mbar_wait(full0 + 8 * (int)(kt % S_STAGES), (uint32_t)(kt / S_STAGES) & 1)) abort_flag = 1;
+        }
+    } else if (lane == 0) {
+        // ---------------- MMA issuer ----------------
+        const uint32_t idesc = make_idesc(BM, n_mma);
+        bool ok = true;
+        for (int64_t kt = 0; kt < ktiles && ok; ++kt) {
+            const int s = (int)(kt % S_STAGES);
+            ok = mbar_wait(full0 + 8 * s, (uint32_t)(kt / S_STAGES) & 1) && !abort_flag;
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a0 = smem_base + s * S_STAGE_BYTES, b0 = a0 + S_A_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < H_BK / 16; ++ks)
+                umma_bf16(tmem_d, make_smem_desc_sw128(a0 + ks * 32), make_smem_desc_sw128(b0 + ks * 32), idesc,
+                          (kt > 0 || ks > 0) ? 1u : 0u);
+            umma_commit(empty0 + 8 * s);
+        }
+        if (!ok) abort_flag = 1;
+        if (ok && ktiles > 0) umma_commit(accum);
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == H_EPI_WARPS) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(H_TMEM_COLS) : "memory");
+    }
+}
+
 }  // namespace tc
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point (the library does not link libcuda)
@@ -683,6 +843,24 @@ grass_status launch_score_bf16(const void* train, int64_t N, int64_t ld_train, c
     if (!make_map(&map_train, train, N, D, ld_train, true, tc::H_BOX_ROWS) ||
         !make_map(&map_test, test, M, D, ld_test, true, tc::H_BOX_ROWS))
         return GRASS_ERR_CUDA;
+    const int out_vec = ((uintptr_t)scores % 16 == 0) && (ld_s % 4 == 0);
+    if (gy == 1 && tuning(GRASS_TUNE_SCORE_BF16_SOLO, 1) != 0) {
+        // one column tile (M <= 256): one thread block per 128 train rows, no cluster
+        const int64_t tiles = (N + tc::BM - 1) / tc::BM;
+        const size_t smem1 = (size_t)tc::S_STAGES * tc::S_STAGE_BYTES + 1024;
+        if (cudaFuncSetAttribute(tc::grass_score_bf16_solo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem1) != cudaSuccess)
+            return GRASS_ERR_CUDA;
+        int64_t splits1 = 1, kt_split1 = 1;
+        if (plan_splits(D, (tiles + 1) / 2, tc::H_BK, &splits1, &kt_split1) != GRASS_OK) return GRASS_ERR_CUDA;
+        if (splits1 > 1 && cudaMemset2DAsync(scores, (size_t)ld_s * sizeof(float), 0, (size_t)M * sizeof(float),
+                                             (size_t)N, st) != cudaSuccess)
+            return GRASS_ERR_CUDA;
+        dim3 grid1((unsigned)tiles, 1, (unsigned)splits1);
+        tc::grass_score_bf16_solo_kernel<<<grid1, tc::S_THREADS, smem1, st>>>(map_train, map_test, N, M, D, kt_split1,
+                                                                              scores, ld_s, out_vec);
+        return launch_status();
+    }
     const size_t smem = (size_t)tc::H_STAGES * tc::H_STAGE_BYTES + 1024;
     if (cudaFuncSetAttribute(tc::grass_score_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)

@@ -41,7 +41,10 @@ def test_to_bf16_is_round_to_nearest_even(G):
 
 @pytest.mark.parametrize("N,M,D", [(300, 70, 264), (128, 128, 64), (1, 1, 8), (513, 256, 4096), (5, 3, 16),
                                    (257, 513, 104), (640, 40, 8), (2048, 256, 4096), (200, 100, 20_000)])
-def test_score_bf16_parity(G, oracle_mod, N, M, D):
+@pytest.mark.parametrize("solo", [1, 0])
+def test_score_bf16_parity(G, oracle_mod, tune, N, M, D, solo):
+    """Both kernels: one thread block per tile (taken for M <= 256) and thread-block pairs (any M)."""
+    tune(score_bf16_solo=solo)
     g = torch.Generator(device="cuda")
     g.manual_seed(N + D)
     pad = 8 * (N % 3)
@@ -61,11 +64,11 @@ def test_score_bf16_forced_splits_and_unsupported_strides(G, oracle_mod, tune):
     tr = torch.randn((260, 1_000), generator=g, device="cuda").to(torch.bfloat16)
     te = torch.randn((90, 1_000), generator=g, device="cuda").to(torch.bfloat16)
     ref, absum = oracle_mod.score(tr.float().cpu().numpy(), te.float().cpu().numpy())
-    for splits in (1, 3, 32):
-        tune(score_splits=splits)
+    for splits, solo in ((1, 1), (3, 1), (32, 1), (1, 0), (3, 0), (32, 0)):
+        tune(score_splits=splits, score_bf16_solo=solo)
         sc = G.grass_score_bf16(tr, te, out=torch.full((260, 90), -1.0, device="cuda"))
         check_close(sc.cpu().numpy(), ref, absum, 1e-4, 1_000 + 72, eps=EPS_TC, what=f"bf16 score, {splits} splits")
-    tune(score_splits=None)
+    tune(score_splits=None, score_bf16_solo=None)
     with pytest.raises(G.GrassError) as e:
         G.grass_score_bf16(tr[:, :996][:, 1:], te[:, :996][:, 1:])          # base not 16-byte aligned
     assert e.value.code == 3
