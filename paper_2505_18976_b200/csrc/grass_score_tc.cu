@@ -228,7 +228,7 @@ grass_score_tc_kernel(const __grid_constant__ CUtensorMap map_train, const __gri
                 const uint32_t off = operand_chunk_offset(r, ch);
                 *reinterpret_cast<uint4*>(base + off) = hi;
                 *reinterpret_cast<uint4*>(base + piece + off) = mid;
-                *reinterpret_cast<uint4*>(base + 2 * piece + off) = lo;
+                if (nprod > 4) *reinterpret_cast<uint4*>(base + 2 * piece + off) = lo;   // no product reads it otherwise
             }
         };
         const uint32_t leader_full0 = map_to_cta(full0, 0);
