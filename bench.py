@@ -174,7 +174,9 @@ class GrassJob:
         self.fetch_bytes_per_launch = cfg.batch * sector_bytes_per_row(self.idx, 4, 64) + cfg.batch * cfg.k * 4
         self.dense_bytes_per_launch = batch_bytes
         self.launches_per_step = self.nbatch
-        self.kernels_per_step = 2 * self.nbatch     # memset + compress kernel per call (upper bound)
+        # one kernel per call: with these shapes the position splits of a row are reduced inside a cluster (config 2)
+        # or a thread block owns a whole row (config 1), so there is no zero-fill before the compress kernel
+        self.kernels_per_step = self.nbatch
         self.dominant = "grass_compress_kernel"
         self.l2 = (f"{self.ncopies} resident batch(es) of {batch_bytes / 1e6:.0f} MB rotated; "
                    + ("input >> L2" if self.ncopies == 1 else L2_FLUSHED))
@@ -245,7 +247,11 @@ class FactJob:
         self.dense_bytes_per_launch = self.dense
         self.launches_per_step = 1
         nb = (cfg.k + 63) // 64
-        self.kernels_per_step = 2 + (1 if self.score else 0) + ((2 + 3 * nb + 4 * nb) if self.precondition else 0)
+        # the grouped call is one kernel when it takes the cluster kernel (few (layer, sample) items: config 3), else a
+        # zero-fill kernel and the streaming kernel (the library's rule: items <= thread-block slots of one wave)
+        items, slots = len(cfg.layers) * cfg.B, 148 * (1 if max(cfg.kin, cfg.kout) > 64 else 2)
+        fact_kernels = 1 if (items <= slots and not fp32_inputs and max(cfg.kin, cfg.kout) <= 128) else 2
+        self.kernels_per_step = fact_kernels + (1 if self.score else 0) + ((2 + 3 * nb + 4 * nb) if self.precondition else 0)
         self.dominant = "factgrass_kernel"
         self.need_flush = self.dense < 4 * L2_BYTES
         self.l2 = L2_FLUSHED if self.need_flush else "inputs >> L2"
