@@ -126,6 +126,9 @@ factgrass_cluster_kernel(const LayerDesc* __restrict__ descs, const __grid_const
 
     cg::cluster_group cluster = cg::this_cluster();
     const uint32_t nc = cluster.num_blocks(), rank = cluster.block_rank();
+    // "I have started": the other half of this barrier is waited for just before the first write into another thread
+    // block's shared memory, which is only defined once that thread block is running (by then everyone has arrived)
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     const LayerDesc& L = descs ? descs[blockIdx.z] : single;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.y;
@@ -254,6 +257,7 @@ factgrass_cluster_kernel(const LayerDesc* __restrict__ descs, const __grid_const
     // exchange: the rows of the partial block go from tensor memory to their owners (zeros where there was no work).
     // Accumulator row a sits in tensor-memory lane a (TM = 128) or lane (a % 16) + 32 * (a / 16) (TM = 64);
     // warp w may read lanes 32 * (w % 4) .. + 31; the two warps that share a lane quarter split the columns.
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");     // every thread block of the cluster runs
     const bool nc_ok = nc == 1 || nc == 2 || nc == 4 || nc == 8;    // the launcher forms no other clusters
     const int rows = TM / (int)(nc_ok ? nc : 1);
     if (nc_ok) {
